@@ -1,0 +1,140 @@
+"""Seeded synthetic inputs shaped like the paper's workloads.
+
+This module only *generates inputs* (random state and activations, model
+shapes); it holds none of the method's arithmetic and is the one module that
+both the CUDA path's callers and the CPU checker's callers may use.
+
+State of W data-parallel workers, each a flat vector of P parameters
+(Section 3.2): slow weights phi ~ N(0, 0.02^2), fast weights
+theta = phi + drift with drift ~ N(0, (1e-3)^2) or Student-t(3) * 1e-3, and
+outer momentum delta ~ N(0, (1e-4)^2).  theta is float32 or bfloat16.
+
+Model shapes follow the paper's Table 3 (hidden size, layers, intermediate
+size) with a 50k-entry tied embedding: P = V*d + L*(4*d*d + 2*d*ff + 2*d) + d.
+"""
+
+from __future__ import annotations
+
+import torch
+
+PHI_STD = 0.02
+DRIFT_STD = 1e-3
+DELTA_STD = 1e-4
+
+# name -> (hidden d, layers L, intermediate ff, heads)   [paper, Table 3]
+MODEL_SHAPES = {
+    "125M": (768, 12, 3072, 12),
+    "1.3B": (2048, 24, 8192, 32),
+    "6.8B": (4096, 32, 16384, 32),
+}
+VOCAB = 50_000
+
+
+def layer_params(d: int, ff: int) -> int:
+    """Parameters of one decoder layer: q,k,v,o projections, a 2-matrix MLP
+    and two norm vectors."""
+    return 4 * d * d + 2 * d * ff + 2 * d
+
+
+def model_params(name: str, vocab: int = VOCAB) -> int:
+    """Flattened parameter count of a whole model (tied embedding + final norm)."""
+    d, L, ff, _ = MODEL_SHAPES[name]
+    return vocab * d + L * layer_params(d, ff) + d
+
+
+def stage_params(name: str, stages: int) -> int:
+    """Parameters of one middle pipeline stage (layers only) when the model
+    is cut into ``stages`` equal runs of layers."""
+    d, L, ff, _ = MODEL_SHAPES[name]
+    assert L % stages == 0
+    return (L // stages) * layer_params(d, ff)
+
+
+def padded_stride(P: int, multiple: int = 64) -> int:
+    """Row stride in elements: P rounded up so that every row starts on a
+    256-byte boundary for 4-byte elements."""
+    return (P + multiple - 1) // multiple * multiple
+
+
+def _gen(device, seed: int) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    return g
+
+
+def _student_t3_(out: torch.Tensor, gen: torch.Generator) -> torch.Tensor:
+    """Fill ``out`` (float32) with Student-t(3) draws: Z / sqrt(chi2_3 / 3)."""
+    z = torch.empty_like(out).normal_(generator=gen)
+    s = torch.zeros_like(out)
+    for _ in range(3):
+        s += torch.empty_like(out).normal_(generator=gen) ** 2
+    out.copy_(z / torch.sqrt(s / 3.0))
+    return out
+
+
+def fill_state_(phi: torch.Tensor, theta: torch.Tensor, delta: torch.Tensor,
+                P: int, seed: int, drift: str = "normal",
+                chunk: int = 1 << 24) -> None:
+    """Fill the first P columns of the [W, stride] state tensors in place.
+
+    Works on CPU or CUDA tensors; large rows are filled in column chunks so
+    the temporaries stay small.  ``theta`` may be float32 or bfloat16.
+    Padding columns (>= P) are left untouched.
+    """
+    W = phi.shape[0]
+    gen = _gen(phi.device, seed)
+    for w in range(W):
+        for c0 in range(0, P, chunk):
+            c1 = min(P, c0 + chunk)
+            p = phi[w, c0:c1]
+            p.normal_(0.0, PHI_STD, generator=gen)
+            d = torch.empty(c1 - c0, dtype=torch.float32, device=phi.device)
+            if drift == "normal":
+                d.normal_(0.0, DRIFT_STD, generator=gen)
+            elif drift == "student_t3":
+                _student_t3_(d, gen).mul_(DRIFT_STD)
+            else:
+                raise ValueError(drift)
+            theta[w, c0:c1].copy_(p + d)          # casts when theta is bfloat16
+            delta[w, c0:c1].normal_(0.0, DELTA_STD, generator=gen)
+
+
+def apply_drift_(phi: torch.Tensor, theta: torch.Tensor, P: int, seed: int,
+                 drift: str = "normal", chunk: int = 1 << 24) -> None:
+    """Stand-in for an inner optimisation phase between two outer steps:
+    theta <- cast(phi + fresh drift)."""
+    W = phi.shape[0]
+    gen = _gen(phi.device, seed)
+    for w in range(W):
+        for c0 in range(0, P, chunk):
+            c1 = min(P, c0 + chunk)
+            d = torch.empty(c1 - c0, dtype=torch.float32, device=phi.device)
+            if drift == "normal":
+                d.normal_(0.0, DRIFT_STD, generator=gen)
+            else:
+                _student_t3_(d, gen).mul_(DRIFT_STD)
+            theta[w, c0:c1].copy_(phi[w, c0:c1] + d)
+
+
+def make_state(W: int, P: int, seed: int, theta_dtype=torch.float32,
+               drift: str = "normal", stride: int | None = None,
+               device="cpu", pad_value: float = 0.0):
+    """Allocate and fill (phi, theta, delta) as [W, stride] tensors."""
+    stride = padded_stride(P, 8) if stride is None else stride
+    phi = torch.full((W, stride), pad_value, dtype=torch.float32, device=device)
+    theta = torch.full((W, stride), pad_value, dtype=theta_dtype, device=device)
+    delta = torch.full((W, stride), pad_value, dtype=torch.float32, device=device)
+    fill_state_(phi, theta, delta, P, seed, drift)
+    return phi, theta, delta
+
+
+def make_acts(boundaries: int, R: int, K: int, E: int, seed: int,
+              dtype=torch.float32, device="cpu") -> torch.Tensor:
+    """Activations at the stage boundaries, [boundaries, R, K, E], N(0, 1)."""
+    gen = _gen(device, seed)
+    out = torch.empty((boundaries, R, K, E), dtype=dtype, device=device)
+    for b in range(boundaries):
+        for r in range(R):
+            out[b, r].copy_(torch.empty((K, E), dtype=torch.float32,
+                                        device=device).normal_(generator=gen))
+    return out
