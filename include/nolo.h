@@ -1,0 +1,220 @@
+/*
+ * nolo.h -- C ABI of the NoLoCo outer synchronisation step and random pipeline
+ * routing for W simulated data-parallel workers resident in one GPU's memory.
+ *
+ * The method is that of "NoLoCo: No-all-reduce Low Communication Training
+ * Method for Large Models" (arXiv 2506.10911): Section 3.2, Eq. 1-3 (outer
+ * step) and Section 3.1 / Algorithm 1 (random pipeline routing).
+ *
+ * Conventions
+ *   - Every function returns an int status: NOLO_OK (0) or a negative NOLO_E*
+ *     code.  Nothing throws; nothing aborts.  nolo_strerror() names a code,
+ *     nolo_last_error() gives the handle's last detailed message.
+ *   - "device" pointers are CUDA device addresses on the device that was
+ *     current when nolo_create() ran; "host" pointers are ordinary (ideally
+ *     page-locked) host addresses.  The library never frees or reallocates a
+ *     caller's buffer; it owns only its small index tables.
+ *   - Calls that enqueue GPU work are asynchronous on the bound stream unless
+ *     stated otherwise.  One handle serves one stream at a time and is not
+ *     thread-safe.
+ *   - Streams are passed as void* holding a cudaStream_t (NULL = default
+ *     stream), so that this header needs no CUDA header.
+ *
+ * Random draws.  The paper only asks for "random" subgroups and routes from a
+ * seed.  This library defines them: element i of a draw of size N gets the
+ * 64-bit key philox4x64-10(counter = (i, boundary, slot, domain),
+ * key = (seed, step)) word 0 (Salmon et al., SC'11), and the permutation lists
+ * the indices in ascending (key, index) order.  domain = 1 for subgroups
+ * (boundary = slot = 0), domain = 2 for routing.
+ */
+#ifndef NOLO_H
+#define NOLO_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NOLO_OK        0
+#define NOLO_EINVAL   (-1)  /* bad argument (range, NULL, n does not divide W, ...) */
+#define NOLO_ESTATE   (-2)  /* a needed nolo_bind_* call has not been made */
+#define NOLO_EALIGN   (-3)  /* pointer or stride violates the alignment rule */
+#define NOLO_ECUDA    (-4)  /* a CUDA runtime call failed; see nolo_last_error() */
+#define NOLO_ENOMEM   (-5)  /* allocation of the handle or its tables failed */
+
+#define NOLO_F32   0        /* element type codes */
+#define NOLO_BF16  1
+
+#define NOLO_MAX_WORKERS 4096
+
+#define NOLO_KERNEL_OUTER 0 /* kernel ids for nolo_timing_read() */
+#define NOLO_KERNEL_ROUTE 1
+
+typedef struct nolo_handle nolo_handle;
+
+/*
+ * Create a context for W workers synchronising in random subgroups of n
+ * (Section 3.2: N model instances, local subgroup of n), each worker a flat
+ * vector of P parameters, in a pipeline of `stages` stages (Section 3.1), with
+ * momentum alpha, outer learning rate beta and local averaging weight gamma
+ * (Eq. 2).
+ *   W      1..NOLO_MAX_WORKERS;  n  1..W and n must divide W (subgroups are a
+ *          disjoint random partition);  P >= 1;  stages >= 1;
+ *   alpha, beta, gamma  finite.
+ * On success *out receives a handle owned by the caller (release it with
+ * nolo_destroy).  On failure *out is NULL (if out itself is non-NULL).
+ * Allocates only index tables (a few KB of device memory) and CUDA events.
+ * Errors: NOLO_EINVAL, NOLO_ENOMEM, NOLO_ECUDA.
+ */
+int nolo_create(int W, int n, int64_t P, int stages,
+                float alpha, float beta, float gamma, nolo_handle** out);
+
+/*
+ * Attach the worker state (borrowed; must stay valid while bound).
+ *   phi    device, float32 [W][row_stride]: slow weights phi_{t,i}
+ *   theta  device, [W][row_stride] of theta_dtype (NOLO_F32 or NOLO_BF16):
+ *          fast weights theta_{t+1,i} left by the inner phase
+ *   delta  device, float32 [W][row_stride]: outer momentum delta_{t-1,i}
+ *   row_stride  elements between consecutive workers' rows; >= P and a
+ *          multiple of 8.  Columns >= P are padding: never read as parameters,
+ *          never written.
+ *   stream cudaStream_t on which all later work of this handle is enqueued.
+ * All three pointers must be 16-byte aligned and the buffers must not overlap.
+ * Errors: NOLO_EINVAL (NULL, bad dtype or stride), NOLO_EALIGN.
+ */
+int nolo_bind_state(nolo_handle* h, void* phi, void* theta, void* delta,
+                    int theta_dtype, int64_t row_stride, void* stream);
+
+/*
+ * One outer step, in place, on the bound state (Section 3.2):
+ *   1. draw the random partition into subgroups from (seed, step);
+ *   2. Delta_j = phi_j - theta_j                        (Eq. 1; the sign that
+ *      makes Eq. 2 move phi toward theta, as the convergence analysis of
+ *      Appendix D and DiLoCo do);
+ *   3. per subgroup G:  mean Delta and mean phi over all n members;
+ *   4. delta_i <- alpha delta_i - beta mean_G(Delta) - gamma (phi_i - mean_G(phi))   (Eq. 2)
+ *      phi_i   <- phi_i + delta_i                                                    (Eq. 3)
+ *      theta_i <- phi_i  (rounded to nearest-even when theta is bfloat16).
+ * float32 arithmetic; every element of every worker is read once and written
+ * once.  Asynchronous.  Errors: NOLO_EINVAL (NULL handle), NOLO_ESTATE (no
+ * state bound), NOLO_ECUDA (launch failure).
+ */
+int nolo_outer_step(nolo_handle* h, uint64_t seed, uint64_t step);
+
+/*
+ * The same step for state that lives in HOST memory: columns are streamed
+ * host -> bound device buffers -> host in chunks, copies overlapped with the
+ * kernel, and the call returns after the last byte is back in host memory
+ * (synchronous).  The device state bound with nolo_bind_state() is used as
+ * the staging area and holds the new state afterwards as well.
+ *   phi_host, theta_host, delta_host  host, same types and [W][host_stride]
+ *          layout as the device buffers (page-locked memory is needed for the
+ *          copies to overlap);  host_stride >= P, in elements.
+ * Errors: as nolo_outer_step, plus NOLO_EINVAL for NULL/short strides.
+ */
+int nolo_outer_step_host(nolo_handle* h, uint64_t seed, uint64_t step,
+                         void* phi_host, void* theta_host, void* delta_host,
+                         int64_t host_stride);
+
+/*
+ * Describe the routed activations (Section 3.1; Algorithm 1).  Each of the
+ * stages-1 boundaries carries M micro-batches of E elements from the W
+ * replicas of one stage to the W replicas of the next; replica r holds
+ * K = M / W micro-batch slots.
+ *   M      number of micro-batches per boundary; a positive multiple of W
+ *   E      elements per micro-batch activation (>= 1)
+ *   act_dtype  NOLO_F32 or NOLO_BF16 (data are moved, never interpreted)
+ *   acts_out   device, [stages-1][W][K][E]: receives the routed activations;
+ *          borrowed; 16-byte aligned; must not overlap the input of nolo_route
+ *   per_microbatch  0: one permutation per (step, boundary), all K slots of a
+ *          replica travel together;  1: every slot k draws its own.
+ * Errors: NOLO_EINVAL, NOLO_EALIGN, NOLO_ENOMEM/NOLO_ECUDA (table allocation).
+ */
+int nolo_bind_route(nolo_handle* h, int M, int64_t E, int act_dtype,
+                    void* acts_out, int per_microbatch);
+
+/*
+ * Forward routing for all stages-1 boundaries (Section 3.1: random
+ * permutations re-drawn every step; Algorithm 1, forward pass): draws
+ * table[b][k][r] = sending replica of stage b whose slot k goes to replica r
+ * of stage b+1 (each table[b][k][:] is a permutation of 0..W-1), then
+ *   acts_out[b][r][k][:] = acts[b][table[b][k][r]][k][:]      (bit copy).
+ *   acts   device, [stages-1][W][K][E], 16-byte aligned, read only.
+ * stages == 1 is a valid no-op.  Uses the stream given to nolo_bind_state,
+ * or the default stream if no state is bound.  Asynchronous.
+ * Errors: NOLO_EINVAL, NOLO_ESTATE (nolo_bind_route not called), NOLO_EALIGN,
+ * NOLO_ECUDA.
+ */
+int nolo_route(nolo_handle* h, uint64_t seed, uint64_t step, const void* acts);
+
+/*
+ * Backward routing (Algorithm 1, backward pass: gradients return along the
+ * path of the forward pass): with the table of (seed, step),
+ *   grads_out[b][table[b][k][r]][k][:] = grads[b][r][k][:].
+ *   grads, grads_out  device, [stages-1][W][K][E], 16-byte aligned, disjoint.
+ * Errors: as nolo_route.
+ */
+int nolo_route_backward(nolo_handle* h, uint64_t seed, uint64_t step,
+                        const void* grads, void* grads_out);
+
+/*
+ * Forward routing for activations in HOST memory: copies acts to a device
+ * staging buffer the caller provides, routes, and copies the result back;
+ * synchronous.
+ *   acts_host, out_host  host, [stages-1][W][K][E]
+ *   acts_dev   device scratch of the same size (input staging); the routed
+ *          result is produced in the acts_out buffer of nolo_bind_route.
+ */
+int nolo_route_host(nolo_handle* h, uint64_t seed, uint64_t step,
+                    const void* acts_host, void* out_host, void* acts_dev);
+
+/*
+ * Copy the subgroup table of the most recent outer step to the host:
+ * perm[W] int32; subgroup g is perm[g*n .. g*n+n-1].  Synchronises the stream.
+ * Errors: NOLO_EINVAL, NOLO_ESTATE (no outer step yet), NOLO_ECUDA.
+ */
+int nolo_get_groups(nolo_handle* h, int32_t* host_out);
+
+/*
+ * Copy the routing table of the most recent route call to the host:
+ * int32 [stages-1][K][W].  Synchronises the stream.
+ * Errors: NOLO_EINVAL, NOLO_ESTATE (no route call yet), NOLO_ECUDA.
+ */
+int nolo_get_route(nolo_handle* h, int32_t* host_out);
+
+/*
+ * Device-time instrumentation.  With enable != 0 every later launch of the
+ * fused outer-step kernel and of the routing copy kernel is bracketed by CUDA
+ * events on the bound stream (up to 4096 launches per kernel between reads).
+ * nolo_timing_read synchronises the stream, returns the summed device time in
+ * milliseconds and the number of bracketed launches of `kernel`
+ * (NOLO_KERNEL_OUTER / NOLO_KERNEL_ROUTE) since the last read, and resets them.
+ */
+int nolo_timing_enable(nolo_handle* h, int enable);
+int nolo_timing_read(nolo_handle* h, int kernel, double* total_ms, int64_t* launches);
+
+/*
+ * Number of kernels this handle has launched since it was created.
+ */
+int nolo_launch_count(nolo_handle* h, int64_t* launches);
+
+/*
+ * Release the handle and its tables.  Bound buffers are not touched.
+ * NULL is accepted.  Waits for the bound stream first.
+ */
+int nolo_destroy(nolo_handle* h);
+
+/* Static text for a status code (never NULL). */
+const char* nolo_strerror(int status);
+
+/* Last detailed error message of this handle ("" if none; never NULL). */
+const char* nolo_last_error(nolo_handle* h);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int nolo_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NOLO_H */

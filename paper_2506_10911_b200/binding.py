@@ -1,0 +1,213 @@
+"""ctypes binding of ``libnolo.so`` (the C ABI declared in ``include/nolo.h``).
+
+Argument marshalling only: the functions here have the names and argument
+order of the C entry points, take ``torch`` tensors (or raw addresses) where
+the C side takes pointers, and raise :class:`NoloError` on a non-zero status.
+There is no fallback: if the shared library is missing, importing this module
+fails.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnolo.so")
+
+NOLO_OK, NOLO_EINVAL, NOLO_ESTATE, NOLO_EALIGN, NOLO_ECUDA, NOLO_ENOMEM = 0, -1, -2, -3, -4, -5
+NOLO_F32, NOLO_BF16 = 0, 1
+NOLO_KERNEL_OUTER, NOLO_KERNEL_ROUTE = 0, 1
+NOLO_MAX_WORKERS = 4096
+
+
+class NoloError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        msg = f"{where}: {_lib.nolo_strerror(status).decode()} ({status})"
+        if detail:
+            msg += f": {detail}"
+        super().__init__(msg)
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2506_10911_b200.build` "
+        "(there is no CPU or PyTorch fallback for the CUDA path)")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+_H = ctypes.c_void_p
+_u64, _i64, _i32, _f32, _vp = ctypes.c_uint64, ctypes.c_int64, ctypes.c_int, ctypes.c_float, ctypes.c_void_p
+
+# name -> argtypes; every entry point of include/nolo.h
+SIGNATURES = {
+    "nolo_create": [_i32, _i32, _i64, _i32, _f32, _f32, _f32, ctypes.POINTER(_H)],
+    "nolo_bind_state": [_H, _vp, _vp, _vp, _i32, _i64, _vp],
+    "nolo_outer_step": [_H, _u64, _u64],
+    "nolo_outer_step_host": [_H, _u64, _u64, _vp, _vp, _vp, _i64],
+    "nolo_bind_route": [_H, _i32, _i64, _i32, _vp, _i32],
+    "nolo_route": [_H, _u64, _u64, _vp],
+    "nolo_route_backward": [_H, _u64, _u64, _vp, _vp],
+    "nolo_route_host": [_H, _u64, _u64, _vp, _vp, _vp],
+    "nolo_get_groups": [_H, _vp],
+    "nolo_get_route": [_H, _vp],
+    "nolo_timing_enable": [_H, _i32],
+    "nolo_timing_read": [_H, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)],
+    "nolo_launch_count": [_H, ctypes.POINTER(_i64)],
+    "nolo_destroy": [_H],
+    "nolo_strerror": [_i32],
+    "nolo_last_error": [_H],
+    "nolo_version": [],
+}
+for _name, _args in SIGNATURES.items():
+    _fn = getattr(_lib, _name)
+    _fn.argtypes = _args
+    _fn.restype = ctypes.c_char_p if _name in ("nolo_strerror", "nolo_last_error") else ctypes.c_int
+
+
+def _ptr(x) -> int:
+    """Address of a torch tensor / numpy array, or an int passed through."""
+    if x is None:
+        return 0
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    return x.data_ptr()
+
+
+def _dtype_code(t) -> int:
+    import torch
+    if t.dtype == torch.float32:
+        return NOLO_F32
+    if t.dtype == torch.bfloat16:
+        return NOLO_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+class Handle:
+    """Owns a ``nolo_handle*``; keeps references to bound tensors alive."""
+
+    def __init__(self, ptr: int, W: int, n: int, P: int, stages: int):
+        self.ptr = ptr
+        self.W, self.n, self.P, self.stages = W, n, P, stages
+        self.K = 0
+        self._keep = {}
+
+    def __del__(self):
+        try:
+            nolo_destroy(self)
+        except Exception:
+            pass
+
+
+def _check(status: int, where: str, h: Handle | None = None):
+    if status != NOLO_OK:
+        detail = _lib.nolo_last_error(h.ptr).decode() if h is not None and h.ptr else ""
+        raise NoloError(status, where, detail)
+
+
+def nolo_create(W: int, n: int, P: int, stages: int, alpha: float, beta: float, gamma: float) -> Handle:
+    out = _H()
+    _check(_lib.nolo_create(W, n, P, stages, alpha, beta, gamma, ctypes.byref(out)), "nolo_create")
+    return Handle(out.value, W, n, P, stages)
+
+
+def nolo_bind_state(h: Handle, phi, theta, delta, stream=None, theta_dtype=None, row_stride=None):
+    """phi/theta/delta: CUDA tensors of shape [W, row_stride]; stream: a
+    ``torch.cuda.Stream`` (default: the current stream)."""
+    import torch
+    if theta_dtype is None:
+        theta_dtype = _dtype_code(theta)
+    if row_stride is None:
+        row_stride = phi.stride(0)
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    sp = stream if isinstance(stream, int) else stream.cuda_stream
+    _check(_lib.nolo_bind_state(h.ptr, _ptr(phi), _ptr(theta), _ptr(delta), theta_dtype, row_stride, sp),
+           "nolo_bind_state", h)
+    h._keep["state"] = (phi, theta, delta, stream)
+
+
+def nolo_outer_step(h: Handle, seed: int, step: int):
+    _check(_lib.nolo_outer_step(h.ptr, seed, step), "nolo_outer_step", h)
+
+
+def nolo_outer_step_host(h: Handle, seed: int, step: int, phi_host, theta_host, delta_host, host_stride=None):
+    if host_stride is None:
+        host_stride = phi_host.stride(0)
+    _check(_lib.nolo_outer_step_host(h.ptr, seed, step, _ptr(phi_host), _ptr(theta_host), _ptr(delta_host),
+                                     host_stride), "nolo_outer_step_host", h)
+
+
+def nolo_bind_route(h: Handle, M: int, E: int, acts_out, per_microbatch: bool = False, act_dtype=None):
+    if act_dtype is None:
+        act_dtype = _dtype_code(acts_out)
+    _check(_lib.nolo_bind_route(h.ptr, M, E, act_dtype, _ptr(acts_out), int(per_microbatch)),
+           "nolo_bind_route", h)
+    h.K = M // h.W
+    h._keep["route"] = acts_out
+
+
+def nolo_route(h: Handle, seed: int, step: int, acts):
+    _check(_lib.nolo_route(h.ptr, seed, step, _ptr(acts)), "nolo_route", h)
+
+
+def nolo_route_backward(h: Handle, seed: int, step: int, grads, grads_out):
+    _check(_lib.nolo_route_backward(h.ptr, seed, step, _ptr(grads), _ptr(grads_out)), "nolo_route_backward", h)
+
+
+def nolo_route_host(h: Handle, seed: int, step: int, acts_host, out_host, acts_dev):
+    _check(_lib.nolo_route_host(h.ptr, seed, step, _ptr(acts_host), _ptr(out_host), _ptr(acts_dev)),
+           "nolo_route_host", h)
+
+
+def nolo_get_groups(h: Handle) -> np.ndarray:
+    out = np.empty(h.W, dtype=np.int32)
+    _check(_lib.nolo_get_groups(h.ptr, out.ctypes.data), "nolo_get_groups", h)
+    return out
+
+
+def nolo_get_route(h: Handle) -> np.ndarray:
+    out = np.empty((max(h.stages - 1, 0), h.K, h.W), dtype=np.int32)
+    _check(_lib.nolo_get_route(h.ptr, out.ctypes.data), "nolo_get_route", h)
+    return out
+
+
+def nolo_timing_enable(h: Handle, enable: bool = True):
+    _check(_lib.nolo_timing_enable(h.ptr, int(enable)), "nolo_timing_enable", h)
+
+
+def nolo_timing_read(h: Handle, kernel: int):
+    """Returns (total milliseconds, launches) since the last read."""
+    ms, cnt = ctypes.c_double(), _i64()
+    _check(_lib.nolo_timing_read(h.ptr, kernel, ctypes.byref(ms), ctypes.byref(cnt)), "nolo_timing_read", h)
+    return ms.value, cnt.value
+
+
+def nolo_launch_count(h: Handle) -> int:
+    cnt = _i64()
+    _check(_lib.nolo_launch_count(h.ptr, ctypes.byref(cnt)), "nolo_launch_count", h)
+    return cnt.value
+
+
+def nolo_destroy(h: Handle):
+    if h is not None and h.ptr:
+        p, h.ptr = h.ptr, 0
+        _lib.nolo_destroy(p)
+        h._keep.clear()
+
+
+def nolo_strerror(status: int) -> str:
+    return _lib.nolo_strerror(status).decode()
+
+
+def nolo_last_error(h: Handle) -> str:
+    return _lib.nolo_last_error(h.ptr if h else None).decode()
+
+
+def nolo_version() -> int:
+    return _lib.nolo_version()

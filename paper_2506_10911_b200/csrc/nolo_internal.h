@@ -1,0 +1,48 @@
+// Internal launch interfaces between the C ABI layer and the kernels.
+// Nothing here is exported.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace nolo {
+
+constexpr int kDomainGroups = 1;  // counter word 3 for subgroup draws
+constexpr int kDomainRoute = 2;   // counter word 3 for routing draws
+
+// Draw `blocks` permutations of 0..N-1 into `table`.
+// Permutation p (0 <= p < boundaries*slots_drawn) has boundary b = p / slots_drawn and
+// slot s = p % slots_drawn, and is written to table[(b*slots_total + k)*N ..] for k = s when
+// slots_drawn == slots_total, or for every k in [0, slots_total) when slots_drawn == 1.
+cudaError_t launch_draw(uint64_t seed, uint64_t step, int domain, int N, int boundaries,
+                        int slots_drawn, int slots_total, int32_t* table, cudaStream_t stream);
+
+struct OuterArgs {
+    float* phi;          // [W][stride]
+    void* theta;         // [W][stride] float or bf16
+    float* delta;        // [W][stride]
+    const int32_t* perm; // [W]; subgroup g = perm[g*n .. g*n+n-1]
+    int64_t stride;      // elements between rows
+    int64_t P;           // columns to process, starting at the pointers given
+    int W, n;
+    int theta_bf16;
+    float alpha, beta, gamma;
+};
+
+// Fused Eq. 1-3 + theta reset over columns [0, P) of the rows (pointers may be pre-offset by
+// a multiple of 8 columns).  One launch.
+cudaError_t launch_outer(const OuterArgs& a, cudaStream_t stream);
+
+struct RouteArgs {
+    const void* in;        // [B][R][K][E]
+    void* out;             // [B][R][K][E]
+    const int32_t* table;  // [B][K][R]
+    int B, R, K;
+    int64_t E;
+    int elem_size;         // bytes
+    int backward;          // 0: out[b][r][k] = in[b][table[b][k][r]][k]; 1: the inverse
+};
+
+cudaError_t launch_route(const RouteArgs& a, cudaStream_t stream);
+
+}  // namespace nolo

@@ -1,0 +1,338 @@
+"""Element-by-element parity of the CUDA path (through the C ABI) with the CPU
+oracle on the same seeded inputs: subgroup and routing tables bit-exact,
+float32 outputs within 1e-7 + 2e-6*|x|, bfloat16 theta within 1 ulp."""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import nolo_oracle as O
+from paper_2506_10911_b200 import synth
+from tests.helpers import assert_bf16_within_1ulp, assert_close_f32, to_np
+
+pytestmark = pytest.mark.gpu
+
+F = float(np.float32(0.5)), float(np.float32(0.7)), float(np.float32(0.5))
+
+
+@pytest.fixture(scope="module")
+def nolo():
+    from paper_2506_10911_b200 import binding
+    return binding
+
+
+def run_both(nolo, W, n, P, seed, step, theta_dtype=torch.float32, stride=None, hp=F,
+             drift="normal", state_seed=0, pad_value=float("nan")):
+    """One outer step on the GPU and in the oracle from the same state.
+    Returns nothing; asserts parity, padding untouched and table equality."""
+    alpha, beta, gamma = hp
+    phi, theta, delta = synth.make_state(W, P, state_seed, theta_dtype, drift, stride, "cpu", pad_value)
+    ins = [to_np(x).copy() for x in (phi, theta, delta)]
+    d_phi, d_theta, d_delta = (x.cuda() for x in (phi, theta, delta))
+    h = nolo.nolo_create(W, n, P, 1, alpha, beta, gamma)
+    nolo.nolo_bind_state(h, d_phi, d_theta, d_delta)
+    nolo.nolo_outer_step(h, seed, step)
+    torch.cuda.synchronize()
+    perm_gpu = nolo.nolo_get_groups(h)
+    nolo.nolo_destroy(h)
+
+    perm = O.draw_groups(seed, step, W, n)
+    assert np.array_equal(perm_gpu, perm), "subgroup table differs from the oracle"
+    bf16 = theta_dtype == torch.bfloat16
+    want = O.outer_step(ins[0][:, :P], ins[1][:, :P], ins[2][:, :P], perm, n, alpha, beta, gamma,
+                        O.THETA_BF16 if bf16 else O.THETA_F32)
+    got = [to_np(x) for x in (d_phi, d_delta, d_theta)]
+    assert_close_f32(got[0][:, :P], want[0], "phi")
+    assert_close_f32(got[1][:, :P], want[1], "delta")
+    if bf16:
+        assert_bf16_within_1ulp(got[2][:, :P], want[2], "theta(bf16)")
+        # theta is the GPU's own phi' rounded to nearest even: exact
+        assert np.array_equal(got[2][:, :P], O.f32_to_bf16_bits(got[0][:, :P]))
+    else:
+        assert_close_f32(got[2][:, :P], want[2], "theta")
+        assert np.array_equal(got[2][:, :P].view(np.uint32), got[0][:, :P].view(np.uint32))
+    # padding columns keep their bits
+    for g, i in zip((got[0], got[2], got[1]), ins):
+        assert np.array_equal(np.ascontiguousarray(g[:, P:]).view(np.uint8),
+                              np.ascontiguousarray(i[:, P:]).view(np.uint8)), "padding was written"
+
+
+# ------------------------------------------------------------------ tables
+
+@pytest.mark.parametrize("W,n", [(1, 1), (2, 2), (4, 2), (8, 4), (16, 2), (32, 8), (128, 8), (128, 128),
+                                 (1000, 5), (4096, 2)])
+def test_subgroup_tables_bit_exact(nolo, W, n):
+    phi, theta, delta = (x.cuda() for x in synth.make_state(W, 8, 0))
+    h = nolo.nolo_create(W, n, 8, 1, *F)
+    nolo.nolo_bind_state(h, phi, theta, delta)
+    for seed, step in [(0, 0), (1, 0), (0, 1), (2**64 - 1, 2**63 + 5), (123456789, 42)]:
+        nolo.nolo_outer_step(h, seed, step)
+        got = nolo.nolo_get_groups(h)
+        assert np.array_equal(got, O.draw_groups(seed, step, W, n))
+    nolo.nolo_destroy(h)
+
+
+# -------------------------------------------------------------- outer step
+
+def test_config1_full(nolo):
+    """W=4, n=2, P=2^20 float32, alpha=.5 beta=.7 gamma=.5, seed 0, step 0."""
+    run_both(nolo, 4, 2, 1 << 20, 0, 0)
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 8, 12, 24])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_group_sizes_and_ragged_tiles(nolo, n, bf16):
+    """P spans several tiles with a ragged tail (not a multiple of 4)."""
+    W = 24
+    dt = torch.bfloat16 if bf16 else torch.float32
+    run_both(nolo, W, n, 5 * 1024 + 3, 7, 3, dt, stride=5 * 1024 + 16)
+
+
+@pytest.mark.parametrize("P", [1, 2, 3, 4, 5, 7, 8, 9, 1023, 1024, 1025, 2047, 2049, 4100])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_small_and_odd_P(nolo, P, bf16):
+    dt = torch.bfloat16 if bf16 else torch.float32
+    run_both(nolo, 4, 2, P, 1, 2, dt)
+    run_both(nolo, 6, 3, P, 1, 2, dt)
+
+
+@pytest.mark.parametrize("hp", [(0.0, 0.0, 1.0), (0.3, 0.7, 0.0), (0.9, 1.0, 1.5), (0.5, 0.7, 0.0)])
+def test_hyperparameter_corners(nolo, hp):
+    hp = tuple(float(np.float32(x)) for x in hp)
+    run_both(nolo, 8, 2, 3000, 5, 5, hp=hp)
+    run_both(nolo, 8, 8, 3000, 5, 5, hp=hp)       # n = W: the DiLoCo case
+
+
+def test_heavy_tailed_drift(nolo):
+    run_both(nolo, 8, 4, 1 << 16, 3, 1, drift="student_t3")
+    run_both(nolo, 32, 8, 1 << 14, 3, 1, drift="student_t3")
+
+
+def test_diloco_reduction_on_gpu(nolo):
+    """n = W, gamma = 0, shared momentum: all replicas take the same global
+    momentum step on the mean outer gradient (Section 3.2)."""
+    W, P = 8, 4096
+    phi, theta, delta = synth.make_state(W, P, 3)
+    delta[:] = delta[0]
+    want_d = 0.3 * delta[0].double() - 0.7 * (phi.double() - theta.double()).mean(0)
+    d_phi, d_theta, d_delta = (x.cuda() for x in (phi, theta, delta))
+    h = nolo.nolo_create(W, W, P, 1, 0.3, 0.7, 0.0)
+    nolo.nolo_bind_state(h, d_phi, d_theta, d_delta)
+    nolo.nolo_outer_step(h, 0, 0)
+    torch.cuda.synchronize()
+    for i in range(W):
+        assert_close_f32(to_np(d_delta[i]), want_d.numpy(), "delta")
+        assert torch.equal(d_delta[i], d_delta[0])
+    nolo.nolo_destroy(h)
+
+
+def test_ten_consecutive_steps_bf16(nolo):
+    """Config-2 pattern at reduced P: 10 outer steps, call k uses (seed k,
+    step k), fresh drift before each; every step is checked from the GPU's own
+    pre-step state, and the final state against a pure-oracle run."""
+    W, n, P = 16, 2, 50_000
+    phi, theta, delta = synth.make_state(W, P, 11, torch.bfloat16)
+    d_phi, d_theta, d_delta = (x.cuda() for x in (phi, theta, delta))
+    o_phi, o_theta, o_delta = (to_np(x).copy() for x in (phi, theta, delta))
+    h = nolo.nolo_create(W, n, P, 1, *F)
+    nolo.nolo_bind_state(h, d_phi, d_theta, d_delta)
+    for k in range(10):
+        if k:
+            synth.apply_drift_(d_phi, d_theta, P, 100 + k)
+            # the pure-oracle trajectory sees the same fast weights (a bf16 rounding flip
+            # in an input would be a different problem, not a rounding difference)
+            o_theta = to_np(d_theta).copy()
+        pre = [to_np(x).copy() for x in (d_phi, d_theta, d_delta)]
+        nolo.nolo_outer_step(h, k, k)
+        torch.cuda.synchronize()
+        perm = O.draw_groups(k, k, W, n)
+        assert np.array_equal(nolo.nolo_get_groups(h), perm)
+        want = O.outer_step(pre[0], pre[1], pre[2], perm, n, *F, O.THETA_BF16)
+        assert_close_f32(to_np(d_phi), want[0], f"phi step {k}")
+        assert_close_f32(to_np(d_delta), want[1], f"delta step {k}")
+        assert_bf16_within_1ulp(to_np(d_theta), want[2], f"theta step {k}")
+        o_phi, o_delta, o_theta = O.outer_step(o_phi, o_theta, o_delta, perm, n, *F, O.THETA_BF16)
+    nolo.nolo_destroy(h)
+    # 10 steps of independent rounding: errors add, so 10x the one-step bound
+    err = np.abs(to_np(d_phi).astype(np.float64) - o_phi)
+    assert (err <= 10 * (1e-7 + 2e-6 * np.abs(o_phi))).all()
+
+
+def test_resume_from_checkpoint_is_exact(nolo):
+    """The draw depends only on (seed, step): a new handle continues exactly."""
+    W, n, P = 8, 2, 10_000
+    phi, theta, delta = synth.make_state(W, P, 5)
+
+    def run(split):
+        a, b, c = (x.clone().cuda() for x in (phi, theta, delta))
+        h = nolo.nolo_create(W, n, P, 1, *F)
+        nolo.nolo_bind_state(h, a, b, c)
+        for k in range(6):
+            if k == split:
+                nolo.nolo_destroy(h)
+                h = nolo.nolo_create(W, n, P, 1, *F)
+                nolo.nolo_bind_state(h, a, b, c)
+            nolo.nolo_outer_step(h, 9, k)
+        torch.cuda.synchronize()
+        nolo.nolo_destroy(h)
+        return a.cpu(), c.cpu()
+
+    a0, c0 = run(-1)
+    a1, c1 = run(3)
+    assert torch.equal(a0, a1) and torch.equal(c0, c1)
+
+
+def test_host_state_path_matches_device_path(nolo):
+    W, n, P = 16, 2, 3_000_001            # several column chunks, ragged tail
+    for dt in (torch.float32, torch.bfloat16):
+        phi, theta, delta = synth.make_state(W, P, 21, dt)
+        stride = phi.stride(0)
+        dev = [x.clone().cuda() for x in (phi, theta, delta)]
+        h = nolo.nolo_create(W, n, P, 1, *F)
+        nolo.nolo_bind_state(h, *dev)
+        nolo.nolo_outer_step(h, 4, 2)
+        torch.cuda.synchronize()
+        want = [x.cpu() for x in dev]
+        host = [x.clone().pin_memory() for x in (phi, theta, delta)]
+        dev2 = [torch.zeros_like(x) for x in dev]
+        nolo.nolo_bind_state(h, *dev2)
+        nolo.nolo_outer_step_host(h, 4, 2, *host, host_stride=stride)
+        for got, w, d2 in zip(host, want, dev2):
+            assert torch.equal(got, w)
+            assert torch.equal(d2.cpu()[:, :P], w[:, :P])
+        nolo.nolo_destroy(h)
+
+
+# ----------------------------------------------------------------- routing
+
+@pytest.mark.parametrize("S,R,K,E,dt,pm", [
+    (2, 4, 2, 2 * 128 * 256, torch.float32, False),      # config 1's routing
+    (4, 8, 4, 4096 + 8, torch.bfloat16, False),
+    (3, 8, 2, 5000, torch.bfloat16, True),
+    (3, 4, 3, 1001, torch.bfloat16, False),              # 2002-byte blocks: element-wise path
+    (2, 16, 1, 333, torch.float32, True),                # 1332-byte blocks: element-wise path
+    (2, 1, 1, 64, torch.float32, False),
+])
+def test_route_bit_exact(nolo, S, R, K, E, dt, pm):
+    acts = synth.make_acts(S - 1, R, K, E, 3, dt)
+    d_acts = acts.cuda()
+    d_out = torch.zeros_like(d_acts)
+    h = nolo.nolo_create(R, 1, 8, S, *F)
+    nolo.nolo_bind_route(h, R * K, E, d_out, pm)
+    for seed, step in [(0, 0), (5, 9)]:
+        nolo.nolo_route(h, seed, step, d_acts)
+        torch.cuda.synchronize()
+        table = O.draw_route(seed, step, S, R, K, pm)
+        assert np.array_equal(nolo.nolo_get_route(h), table)
+        want = O.route_forward(to_np(acts), table)
+        assert np.array_equal(to_np(d_out), want)
+        # gradients return along the same path
+        d_back = torch.zeros_like(d_acts)
+        nolo.nolo_route_backward(h, seed, step, d_out, d_back)
+        torch.cuda.synchronize()
+        assert np.array_equal(to_np(d_back), O.route_backward(want, table))
+        assert torch.equal(d_back.view(torch.uint8), d_acts.view(torch.uint8))
+    nolo.nolo_destroy(h)
+
+
+def test_route_single_stage_is_a_noop(nolo):
+    h = nolo.nolo_create(4, 2, 8, 1, *F)
+    out = torch.zeros(8, device="cuda")
+    nolo.nolo_bind_route(h, 4, 2, out)
+    nolo.nolo_route(h, 0, 0, torch.ones(8, device="cuda"))
+    torch.cuda.synchronize()
+    assert not out.any()
+    nolo.nolo_destroy(h)
+
+
+def test_route_host_path(nolo):
+    S, R, K, E = 3, 4, 2, 4096
+    acts = synth.make_acts(S - 1, R, K, E, 8, torch.bfloat16)
+    h = nolo.nolo_create(R, 2, 8, S, *F)
+    d_out = torch.zeros_like(acts, device="cuda")
+    stage = torch.zeros_like(acts, device="cuda")
+    nolo.nolo_bind_route(h, R * K, E, d_out)
+    src, dst = acts.pin_memory(), torch.zeros_like(acts).pin_memory()
+    nolo.nolo_route_host(h, 2, 3, src, dst, stage)
+    want = O.route_forward(to_np(acts), O.draw_route(2, 3, S, R, K))
+    assert np.array_equal(to_np(dst), want)
+    nolo.nolo_destroy(h)
+
+
+# ----------------------------------------------------- boundary behaviour
+
+def test_error_codes(nolo):
+    h = nolo.nolo_create(4, 2, 100, 2, *F)
+    with pytest.raises(nolo.NoloError) as e:
+        nolo.nolo_outer_step(h, 0, 0)
+    assert e.value.status == nolo.NOLO_ESTATE
+    with pytest.raises(nolo.NoloError) as e:
+        nolo.nolo_get_groups(h)
+    assert e.value.status == nolo.NOLO_ESTATE
+    with pytest.raises(nolo.NoloError) as e:
+        nolo.nolo_route(h, 0, 0, torch.zeros(8, device="cuda"))
+    assert e.value.status == nolo.NOLO_ESTATE
+    big = torch.zeros(3 * 4 * 104 + 16, device="cuda")
+    ok = [big[i * 416:(i + 1) * 416].view(4, 104) for i in range(3)]
+    with pytest.raises(nolo.NoloError) as e:                    # stride < P
+        nolo.nolo_bind_state(h, *ok, row_stride=96)
+    assert e.value.status == nolo.NOLO_EINVAL
+    with pytest.raises(nolo.NoloError) as e:                    # stride not a multiple of 8
+        nolo.nolo_bind_state(h, *ok, row_stride=100)
+    assert e.value.status == nolo.NOLO_EALIGN
+    with pytest.raises(nolo.NoloError) as e:                    # misaligned pointer
+        nolo.nolo_bind_state(h, big[1:417].view(4, 104), ok[1], ok[2])
+    assert e.value.status == nolo.NOLO_EALIGN
+    with pytest.raises(nolo.NoloError) as e:                    # overlapping buffers
+        nolo.nolo_bind_state(h, ok[0], ok[0], ok[2])
+    assert e.value.status == nolo.NOLO_EINVAL
+    assert "overlap" in nolo.nolo_last_error(h)
+    with pytest.raises(nolo.NoloError) as e:                    # M not a multiple of W
+        nolo.nolo_bind_route(h, 6, 16, torch.zeros(64, device="cuda"))
+    assert e.value.status == nolo.NOLO_EINVAL
+    out = torch.zeros(4 * 16, device="cuda")
+    nolo.nolo_bind_route(h, 4, 16, out)
+    with pytest.raises(nolo.NoloError) as e:                    # input aliases output
+        nolo.nolo_route(h, 0, 0, out)
+    assert e.value.status == nolo.NOLO_EINVAL
+    nolo.nolo_bind_state(h, *ok)                                # the handle is still usable
+    nolo.nolo_outer_step(h, 0, 0)
+    torch.cuda.synchronize()
+    nolo.nolo_destroy(h)
+
+
+def test_timing_and_launch_count(nolo):
+    W, n, P = 4, 2, 1 << 16
+    dev = [x.cuda() for x in synth.make_state(W, P, 0)]
+    h = nolo.nolo_create(W, n, P, 2, *F)
+    nolo.nolo_bind_state(h, *dev)
+    acts = torch.zeros(1, W, 1, 1024, device="cuda")
+    out = torch.zeros_like(acts)
+    nolo.nolo_bind_route(h, W, 1024, out)
+    nolo.nolo_timing_enable(h, True)
+    for k in range(5):
+        nolo.nolo_outer_step(h, 0, k)
+        nolo.nolo_route(h, 0, k, acts)
+    ms, cnt = nolo.nolo_timing_read(h, nolo.NOLO_KERNEL_OUTER)
+    assert cnt == 5 and 0 < ms < 1000
+    ms, cnt = nolo.nolo_timing_read(h, nolo.NOLO_KERNEL_ROUTE)
+    assert cnt == 5 and 0 < ms < 1000
+    assert nolo.nolo_timing_read(h, nolo.NOLO_KERNEL_OUTER)[1] == 0
+    assert nolo.nolo_launch_count(h) == 20       # (draw + step) + (draw + copy) per iteration
+    nolo.nolo_destroy(h)
+
+
+def test_non_default_stream(nolo):
+    W, n, P = 4, 2, 10_000
+    phi, theta, delta = synth.make_state(W, P, 2)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        dev = [x.cuda() for x in (phi, theta, delta)]
+        h = nolo.nolo_create(W, n, P, 1, *F)
+        nolo.nolo_bind_state(h, *dev, stream=s)
+        nolo.nolo_outer_step(h, 1, 1)
+    s.synchronize()
+    perm = O.draw_groups(1, 1, W, n)
+    want = O.outer_step(to_np(phi), to_np(theta), to_np(delta), perm, n, *F)
+    assert_close_f32(to_np(dev[0]), want[0], "phi")
+    nolo.nolo_destroy(h)
