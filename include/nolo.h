@@ -47,6 +47,7 @@ extern "C" {
 #define NOLO_BF16  1
 
 #define NOLO_MAX_WORKERS 4096
+#define NOLO_STATIC_MAX_WORKERS 1024   /* limit of nolo_outer_step_static */
 
 #define NOLO_KERNEL_OUTER 0 /* kernel ids for nolo_timing_read() */
 #define NOLO_KERNEL_ROUTE 1
@@ -101,6 +102,35 @@ int nolo_bind_state(nolo_handle* h, void* phi, void* theta, void* delta,
  * state bound), NOLO_ECUDA (launch failure).
  */
 int nolo_outer_step(nolo_handle* h, uint64_t seed, uint64_t step);
+
+/*
+ * (No counterpart in the paper: this is a packaging variant of nolo_outer_step.)
+ *
+ * The same outer step for callers that must not allocate memory: a trainer whose own memory pool
+ * took the whole device at start-up, a process held to a fixed device-memory budget, or a
+ * latency-critical loop that cannot afford the device-wide synchronisation inside
+ * cudaMalloc / cudaFree.  It needs no handle and calls no cudaMalloc, cudaFree or other
+ * allocating routine, on device or host.  The subgroup table, which the handle-based path keeps
+ * in memory from cudaMalloc, lives here in a fixed array inside the library's device image:
+ * NOLO_STATIC_MAX_WORKERS int32 entries = 4 KiB, held by every GPU that loads the library until
+ * the process exits.
+ *   W, n, P, alpha, beta, gamma   as for nolo_create, but W <= NOLO_STATIC_MAX_WORKERS; a larger
+ *          W is rejected with NOLO_EINVAL and a message naming the limit
+ *   phi, theta, delta, theta_dtype, row_stride, stream   as for nolo_bind_state (device
+ *          pointers, borrowed, updated in place)
+ *   seed, step   as for nolo_outer_step; results are bit-identical to it
+ *   err, err_len  optional host buffer that receives a message when the status is not NOLO_OK
+ * The first call on each device looks up the array's device address (that device must be
+ * current, as it must for every call); make that first call before any stream capture begins.
+ * All calls on a device share the one table and each call overwrites the entries it uses, so
+ * nothing needs clearing between calls -- but two calls whose GPU work overlaps (different
+ * streams, no ordering between them) race on the table and give undefined subgroups: order them.
+ * Asynchronous.  Errors: NOLO_EINVAL, NOLO_EALIGN, NOLO_ECUDA.
+ */
+int nolo_outer_step_static(int W, int n, int64_t P, float alpha, float beta, float gamma,
+                           void* phi, void* theta, void* delta, int theta_dtype,
+                           int64_t row_stride, uint64_t seed, uint64_t step, void* stream,
+                           char* err, int err_len);
 
 /*
  * The same step for state that lives in HOST memory: columns are streamed

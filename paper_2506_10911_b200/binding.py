@@ -21,6 +21,7 @@ NOLO_OK, NOLO_EINVAL, NOLO_ESTATE, NOLO_EALIGN, NOLO_ECUDA, NOLO_ENOMEM = 0, -1,
 NOLO_F32, NOLO_BF16 = 0, 1
 NOLO_KERNEL_OUTER, NOLO_KERNEL_ROUTE = 0, 1
 NOLO_MAX_WORKERS = 4096
+NOLO_STATIC_MAX_WORKERS = 1024
 
 
 class NoloError(RuntimeError):
@@ -47,6 +48,8 @@ SIGNATURES = {
     "nolo_create": [_i32, _i32, _i64, _i32, _f32, _f32, _f32, ctypes.POINTER(_H)],
     "nolo_bind_state": [_H, _vp, _vp, _vp, _i32, _i64, _vp],
     "nolo_outer_step": [_H, _u64, _u64],
+    "nolo_outer_step_static": [_i32, _i32, _i64, _f32, _f32, _f32, _vp, _vp, _vp, _i32, _i64, _u64, _u64, _vp,
+                               ctypes.c_char_p, _i32],
     "nolo_outer_step_host": [_H, _u64, _u64, _vp, _vp, _vp, _i64],
     "nolo_bind_route": [_H, _i32, _i64, _i32, _vp, _i32],
     "nolo_route": [_H, _u64, _u64, _vp],
@@ -134,6 +137,28 @@ def nolo_bind_state(h: Handle, phi, theta, delta, stream=None, theta_dtype=None,
 
 def nolo_outer_step(h: Handle, seed: int, step: int):
     _check(_lib.nolo_outer_step(h.ptr, seed, step), "nolo_outer_step", h)
+
+
+def nolo_outer_step_static(W: int, n: int, P: int, alpha: float, beta: float, gamma: float,
+                           phi, theta, delta, seed: int, step: int, stream=None,
+                           theta_dtype=None, row_stride=None):
+    """Outer step without a handle and without any allocation (for callers whose device memory
+    is entirely owned by their own pool, or who may not call cudaMalloc for other reasons).
+    W is limited to NOLO_STATIC_MAX_WORKERS.  Call it once on each device before any stream
+    capture; do not let two calls overlap on the GPU."""
+    import torch
+    if theta_dtype is None:
+        theta_dtype = _dtype_code(theta)
+    if row_stride is None:
+        row_stride = phi.stride(0)
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    sp = stream if isinstance(stream, int) else stream.cuda_stream
+    err = ctypes.create_string_buffer(256)
+    status = _lib.nolo_outer_step_static(W, n, P, alpha, beta, gamma, _ptr(phi), _ptr(theta), _ptr(delta),
+                                         theta_dtype, row_stride, seed, step, sp, err, len(err))
+    if status != NOLO_OK:
+        raise NoloError(status, "nolo_outer_step_static", err.value.decode())
 
 
 def nolo_outer_step_host(h: Handle, seed: int, step: int, phi_host, theta_host, delta_host, host_stride=None):
