@@ -15,7 +15,9 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libnolo.so")
+# NOLO_LIBRARY may name another build of the same library (e.g. one compiled with other tile
+# parameters); by default the library sits next to this file.
+LIB_PATH = os.environ.get("NOLO_LIBRARY") or os.path.join(_HERE, "libnolo.so")
 
 NOLO_OK, NOLO_EINVAL, NOLO_ESTATE, NOLO_EALIGN, NOLO_ECUDA, NOLO_ENOMEM = 0, -1, -2, -3, -4, -5
 NOLO_F32, NOLO_BF16 = 0, 1

@@ -12,13 +12,36 @@
 //   theta_i' = phi_i'   (start of the next inner phase)
 #include "nolo_internal.h"
 
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
+
+namespace cg = cooperative_groups;
 
 namespace nolo {
 
 namespace {
 
-constexpr int kThreads = 256;
+// Launch shape.  One CTA = kThreads threads; a thread of the register-resident kernel handles
+// ITEMS quads for all members of its subgroup.  The defaults were chosen by measurement on B200.
+#ifndef NOLO_THREADS
+#define NOLO_THREADS 256
+#endif
+#ifndef NOLO_MIN_BLOCKS
+#define NOLO_MIN_BLOCKS 1
+#endif
+#ifndef NOLO_ITEMS_N1
+#define NOLO_ITEMS_N1 4
+#endif
+#ifndef NOLO_ITEMS_N2
+#define NOLO_ITEMS_N2 2
+#endif
+#ifndef NOLO_ITEMS_N4
+#define NOLO_ITEMS_N4 1
+#endif
+#ifndef NOLO_ITEMS_N8
+#define NOLO_ITEMS_N8 1
+#endif
+constexpr int kThreads = NOLO_THREADS;
 
 struct KArgs {
     float* phi;
@@ -45,6 +68,25 @@ __device__ __forceinline__ float4 load_theta4(const __nv_bfloat16* row, int64_t 
     r.w = __uint_as_float(v.y & 0xffff0000u);
     return r;
 }
+// Raw (unconverted) loads, so that the conversion sits with the arithmetic and never between loads.
+__device__ __forceinline__ float4 load_theta_raw(const float* row, int64_t q) {
+    return __ldcs(reinterpret_cast<const float4*>(row) + q);
+}
+__device__ __forceinline__ uint2 load_theta_raw(const __nv_bfloat16* row, int64_t q) {
+    return __ldcs(reinterpret_cast<const uint2*>(row) + q);
+}
+__device__ __forceinline__ float4 widen(float4 v) { return v; }
+__device__ __forceinline__ float4 widen(uint2 v) {
+    float4 r;
+    r.x = __uint_as_float(v.x << 16);
+    r.y = __uint_as_float(v.x & 0xffff0000u);
+    r.z = __uint_as_float(v.y << 16);
+    r.w = __uint_as_float(v.y & 0xffff0000u);
+    return r;
+}
+template <typename ThetaT> struct ThetaRaw { using type = float4; };
+template <> struct ThetaRaw<__nv_bfloat16> { using type = uint2; };
+
 __device__ __forceinline__ void store_theta4(float* row, int64_t q, float4 v) {
     __stcs(reinterpret_cast<float4*>(row) + q, v);
 }
@@ -103,7 +145,7 @@ __device__ void scalar_tail(const KArgs& a, int g) {
 // N members: phi_j stays in registers between the reduction and the update, so nothing is read
 // twice.  All loads of a thread are issued before the first use to keep many bytes in flight.
 template <int N, typename ThetaT, int ITEMS>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, NOLO_MIN_BLOCKS)
 outer_step_reg_kernel(const KArgs a) {
     const int g = blockIdx.y;
     const int64_t full_quads = a.P >> 2;
@@ -161,6 +203,145 @@ outer_step_reg_kernel(const KArgs a) {
     if ((a.P & 3) && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) scalar_tail<ThetaT>(a, g);
 }
 
+// ---- large subgroups (8 < n <= 512): members split across warps, CTAs and a cluster --------
+//
+// Holding phi of every member of a tile in registers costs n x 512 bytes per 32 quads, and the
+// kernel only streams at full bandwidth while more than one CTA fits on an SM (one CTA's loads
+// must overlap another's barrier and stores).  So a CTA takes at most 64 members: warp w of its
+// G <= 8 warps holds up to 8 members, w*MPW .. w*MPW+MPW-1 of the CTA's share, for the same 32
+// quads (each member row is read in coalesced 512-byte segments), and a larger subgroup is spread
+// over a thread-block cluster of C = 2, 4 or 8 CTAs that work on the same tile.  Partial sums meet
+// in shared memory (warps of a CTA) and then in distributed shared memory (CTAs of the cluster);
+// both are added in a fixed order, so the result is deterministic and identical in every CTA.
+// As in the small-n kernel every element is read once and written once.  The CTA shape (64
+// members, 8 per warp) measured best on B200 among 32/64/128 members and 4/8 per warp.
+#ifndef NOLO_SPLIT_CTA_MEMBERS
+#define NOLO_SPLIT_CTA_MEMBERS 64     // members one CTA holds (larger subgroups use a cluster)
+#endif
+#ifndef NOLO_SPLIT_PREF
+#define NOLO_SPLIT_PREF 8             // members per warp aimed at when a CTA has more than 16 members
+#endif
+constexpr int kSplitMaxCluster = 8;
+constexpr int kSplitMembersPerCta = NOLO_SPLIT_CTA_MEMBERS;
+constexpr int kSplitMaxWarps = 16;
+
+// Launch bounds: MAXW warps per CTA; registers per thread capped so that several CTAs fit an SM.
+template <int MPW, int MAXW>
+struct SplitShape {
+    static constexpr int kRegs = MPW <= 4 ? 80 : 128;
+    static constexpr int kMinBlocks = (65536 / (MAXW * 32 * kRegs)) > 0 ? (65536 / (MAXW * 32 * kRegs)) : 1;
+};
+
+template <int MPW, typename ThetaT, bool CLUSTER, int MAXW>
+__global__ void __launch_bounds__(MAXW * 32, SplitShape<MPW, MAXW>::kMinBlocks)
+outer_step_split_kernel(const KArgs a, int members_per_cta) {
+    __shared__ float4 part_D[kSplitMaxWarps][32];
+    __shared__ float4 part_P[kSplitMaxWarps][32];
+    __shared__ float4 cta_D[32];
+    __shared__ float4 cta_P[32];
+    const int G = blockDim.x >> 5;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = blockIdx.y;
+    const int n = a.n;
+    int C = 1, rank = 0;
+    if (CLUSTER) {
+        cg::cluster_group cluster = cg::this_cluster();
+        C = (int)cluster.num_blocks();
+        rank = (int)cluster.block_rank();
+    }
+    const int64_t tile = CLUSTER ? (int64_t)(blockIdx.x / C) : (int64_t)blockIdx.x;
+    const int64_t q = tile * 32 + lane;
+    const bool ok = q < (a.P >> 2);
+    const int j_begin = rank * members_per_cta;
+    const int j_end = min(n, j_begin + members_per_cta);
+    const int j0 = j_begin + warp * MPW;
+
+    int row[MPW];
+#pragma unroll
+    for (int m = 0; m < MPW; ++m) row[m] = (j0 + m < j_end) ? __ldg(a.perm + g * n + j0 + m) : -1;
+
+    float4 phi[MPW], dlt[MPW];
+    float4 sD = make_float4(0.f, 0.f, 0.f, 0.f), sP = sD;
+    if (ok) {
+        typename ThetaRaw<ThetaT>::type raw[MPW];
+#pragma unroll
+        for (int m = 0; m < MPW; ++m) {
+            if (row[m] >= 0) {
+                const int64_t off = (int64_t)row[m] * a.stride;
+                phi[m] = __ldcs(reinterpret_cast<const float4*>(a.phi + off) + q);
+                raw[m] = load_theta_raw(static_cast<const ThetaT*>(a.theta) + off, q);
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < MPW; ++m) {
+            if (row[m] >= 0)
+                dlt[m] = __ldcs(reinterpret_cast<const float4*>(a.delta + (int64_t)row[m] * a.stride) + q);
+        }
+#pragma unroll
+        for (int m = 0; m < MPW; ++m) {
+            if (row[m] >= 0) {
+                const float4 t = widen(raw[m]);
+                sD.x += phi[m].x - t.x;  sP.x += phi[m].x;
+                sD.y += phi[m].y - t.y;  sP.y += phi[m].y;
+                sD.z += phi[m].z - t.z;  sP.z += phi[m].z;
+                sD.w += phi[m].w - t.w;  sP.w += phi[m].w;
+            }
+        }
+    }
+    part_D[warp][lane] = sD;
+    part_P[warp][lane] = sP;
+    __syncthreads();
+    // sum over the warps of this CTA, in warp order
+    sD = part_D[0][lane];
+    sP = part_P[0][lane];
+    for (int w = 1; w < G; ++w) {
+        const float4 d = part_D[w][lane], p = part_P[w][lane];
+        sD.x += d.x; sD.y += d.y; sD.z += d.z; sD.w += d.w;
+        sP.x += p.x; sP.y += p.y; sP.z += p.z; sP.w += p.w;
+    }
+    if (CLUSTER) {
+        cg::cluster_group cluster = cg::this_cluster();
+        if (warp == 0) {
+            cta_D[lane] = sD;
+            cta_P[lane] = sP;
+        }
+        cluster.sync();                       // every CTA's sums are published
+        // sum over the CTAs of the cluster, in rank order, through distributed shared memory
+        const float4* rD = cluster.map_shared_rank(cta_D, 0);
+        const float4* rP = cluster.map_shared_rank(cta_P, 0);
+        sD = rD[lane];
+        sP = rP[lane];
+        for (int c = 1; c < C; ++c) {
+            rD = cluster.map_shared_rank(cta_D, c);
+            rP = cluster.map_shared_rank(cta_P, c);
+            const float4 d = rD[lane], p = rP[lane];
+            sD.x += d.x; sD.y += d.y; sD.z += d.z; sD.w += d.w;
+            sP.x += p.x; sP.y += p.y; sP.z += p.z; sP.w += p.w;
+        }
+        cluster.barrier_arrive();             // this CTA no longer reads its peers' shared memory
+    }
+    if (ok) {
+        const float4 mP = make_float4(sP.x * a.inv_n, sP.y * a.inv_n, sP.z * a.inv_n, sP.w * a.inv_n);
+#pragma unroll
+        for (int m = 0; m < MPW; ++m) {
+            if (row[m] >= 0) {
+                const int64_t off = (int64_t)row[m] * a.stride;
+                float4 d, p;
+                p.x = update1(phi[m].x, dlt[m].x, sD.x, mP.x, a, &d.x);
+                p.y = update1(phi[m].y, dlt[m].y, sD.y, mP.y, a, &d.y);
+                p.z = update1(phi[m].z, dlt[m].z, sD.z, mP.z, a, &d.z);
+                p.w = update1(phi[m].w, dlt[m].w, sD.w, mP.w, a, &d.w);
+                __stcs(reinterpret_cast<float4*>(a.phi + off) + q, p);
+                __stcs(reinterpret_cast<float4*>(a.delta + off) + q, d);
+                store_theta4(static_cast<ThetaT*>(a.theta) + off, q, p);
+            }
+        }
+    }
+    if ((a.P & 3) && rank == 0 && tile == (int64_t)(gridDim.x / C) - 1 && threadIdx.x == 0)
+        scalar_tail<ThetaT>(a, g);
+    if (CLUSTER) cg::this_cluster().barrier_wait();   // peers may still be reading this CTA's sums
+}
+
 // ---- any subgroup size: two passes over the members -------------------------------------
 //
 // Pass 1 accumulates the two sums; pass 2 re-reads phi_i (the tile was just touched, so this is
@@ -216,6 +397,32 @@ cudaError_t launch_reg(const KArgs& k, int groups, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
+template <int MPW, typename ThetaT, int MAXW>
+cudaError_t launch_split(const KArgs& k, int groups, int warps, int cluster, int members_per_cta,
+                         cudaStream_t stream) {
+    const int64_t quads = (k.P + 3) >> 2;
+    const int64_t tiles = (quads + 31) / 32;
+    if (tiles * cluster > 0x7fffffffll) return cudaErrorInvalidConfiguration;
+    if (cluster == 1) {
+        dim3 grid((unsigned)tiles, (unsigned)groups);
+        outer_step_split_kernel<MPW, ThetaT, false, MAXW><<<grid, warps * 32, 0, stream>>>(k, members_per_cta);
+        return cudaGetLastError();
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(tiles * cluster), (unsigned)groups);
+    cfg.blockDim = dim3(warps * 32);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = cluster;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, outer_step_split_kernel<MPW, ThetaT, true, MAXW>, k, members_per_cta);
+}
+
 template <typename ThetaT>
 cudaError_t launch_any(const KArgs& k, int groups, cudaStream_t stream) {
     const int64_t quads = (k.P + 3) >> 2;
@@ -229,12 +436,35 @@ cudaError_t launch_any(const KArgs& k, int groups, cudaStream_t stream) {
 template <typename ThetaT>
 cudaError_t dispatch(const KArgs& k, int groups, cudaStream_t stream) {
     switch (k.n) {
-        case 1:  return launch_reg<1, ThetaT, 4>(k, groups, stream);
-        case 2:  return launch_reg<2, ThetaT, 2>(k, groups, stream);
-        case 4:  return launch_reg<4, ThetaT, 1>(k, groups, stream);
-        case 8:  return launch_reg<8, ThetaT, 1>(k, groups, stream);
-        default: return launch_any<ThetaT>(k, groups, stream);
+        case 1:  return launch_reg<1, ThetaT, NOLO_ITEMS_N1>(k, groups, stream);
+        case 2:  return launch_reg<2, ThetaT, NOLO_ITEMS_N2>(k, groups, stream);
+        case 3:  return launch_reg<3, ThetaT, 1>(k, groups, stream);
+        case 4:  return launch_reg<4, ThetaT, NOLO_ITEMS_N4>(k, groups, stream);
+        case 5:  return launch_reg<5, ThetaT, 1>(k, groups, stream);
+        case 6:  return launch_reg<6, ThetaT, 1>(k, groups, stream);
+        case 7:  return launch_reg<7, ThetaT, 1>(k, groups, stream);
+        case 8:  return launch_reg<8, ThetaT, NOLO_ITEMS_N8>(k, groups, stream);
+        default: break;
     }
+    if (k.n <= kSplitMembersPerCta * kSplitMaxCluster) {
+        int cluster = 1;
+        while (cluster * kSplitMembersPerCta < k.n) cluster *= 2;          // 1, 2, 4 or 8 CTAs
+        const int per_cta = (k.n + cluster - 1) / cluster;                 // members per CTA
+        const int pref = per_cta > 16 ? NOLO_SPLIT_PREF : 4;               // members per warp aimed at
+        const int G = (per_cta + pref - 1) / pref;
+        const int mpw = (per_cta + G - 1) / G;
+        constexpr int MAXW = (kSplitMembersPerCta + NOLO_SPLIT_PREF - 1) / NOLO_SPLIT_PREF;
+        static_assert(MAXW <= kSplitMaxWarps && MAXW >= 4, "CTA shape out of range");
+        switch (mpw) {
+#define NOLO_SPLIT_CASE(M) \
+    case M: return launch_split<M, ThetaT, MAXW>(k, groups, G, cluster, per_cta, stream);
+            NOLO_SPLIT_CASE(1) NOLO_SPLIT_CASE(2) NOLO_SPLIT_CASE(3) NOLO_SPLIT_CASE(4)
+            NOLO_SPLIT_CASE(5) NOLO_SPLIT_CASE(6) NOLO_SPLIT_CASE(7) NOLO_SPLIT_CASE(8)
+#undef NOLO_SPLIT_CASE
+            default: break;
+        }
+    }
+    return launch_any<ThetaT>(k, groups, stream);            // n > 256
 }
 
 }  // namespace

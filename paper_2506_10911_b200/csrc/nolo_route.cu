@@ -10,9 +10,12 @@ namespace nolo {
 
 namespace {
 
+#ifndef NOLO_ROUTE_ILP
+#define NOLO_ROUTE_ILP 4
+#endif
 constexpr int kThreads = 256;
-constexpr int kVecPerThread = 4;
-constexpr int kTileVecs = kThreads * kVecPerThread;   // 16 KiB per tile
+constexpr int kVecPerThread = NOLO_ROUTE_ILP;
+constexpr int kTileVecs = kThreads * kVecPerThread;   // vectors per tile
 
 struct Blocks {
     int64_t src, dst;   // block indices into [B][R][K]
@@ -31,7 +34,7 @@ __device__ __forceinline__ Blocks resolve(int64_t blk, const int32_t* __restrict
     return o;
 }
 
-// Blocks of `vecs` 16-byte vectors each; tiles of kTileVecs vectors; CTAs stride over tiles.
+// Blocks of `vecs` 16-byte vectors each; tiles of kTileVecs vectors; one tile per CTA.
 __global__ void __launch_bounds__(kThreads)
 route_copy16_kernel(const uint4* __restrict__ in, uint4* __restrict__ out,
                     const int32_t* __restrict__ table, int R, int K, int64_t vecs,
@@ -76,12 +79,11 @@ route_copy_elem_kernel(const T* __restrict__ in, T* __restrict__ out, const int3
     }
 }
 
-int resident_grid(int64_t total_tiles) {
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess)
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int64_t want = (int64_t)sms * 8;   // 8 CTAs of 256 threads fill an SM
-    return (int)(total_tiles < want ? total_tiles : want);
+// One CTA per tile (a one-shot grid streams through memory in address order, which measured
+// about 10 % faster on B200 than a resident grid striding over the tiles); the kernels still loop
+// so that a tile count beyond the grid limit stays correct.
+int tile_grid(int64_t total_tiles) {
+    return (int)(total_tiles < 0x7fffffffll ? total_tiles : 0x7fffffffll);
 }
 
 }  // namespace
@@ -94,13 +96,13 @@ cudaError_t launch_route(const RouteArgs& a, cudaStream_t stream) {
         const int64_t vecs = bytes / 16;
         const int64_t tpb = (vecs + kTileVecs - 1) / kTileVecs;
         const int64_t total = tpb * blocks;
-        route_copy16_kernel<<<resident_grid(total), kThreads, 0, stream>>>(
+        route_copy16_kernel<<<tile_grid(total), kThreads, 0, stream>>>(
             static_cast<const uint4*>(a.in), static_cast<uint4*>(a.out), a.table, a.R, a.K, vecs, tpb,
             total, a.backward);
     } else {
         const int64_t tpb = (a.E + kTileVecs - 1) / kTileVecs;
         const int64_t total = tpb * blocks;
-        const int grid = resident_grid(total);
+        const int grid = tile_grid(total);
         if (a.elem_size == 4)
             route_copy_elem_kernel<uint32_t><<<grid, kThreads, 0, stream>>>(
                 static_cast<const uint32_t*>(a.in), static_cast<uint32_t*>(a.out), a.table, a.R, a.K,

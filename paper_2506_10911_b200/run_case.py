@@ -39,7 +39,9 @@ def main(argv=None):
                     "per-chunk normal/drift recipe (timing only; values do not affect the kernels' time)")
     args = ap.parse_args(argv)
 
-    build.build()
+    import os
+    if not os.environ.get("NOLO_LIBRARY"):
+        build.build()
     from . import binding as nolo
 
     P = args.P

@@ -88,6 +88,18 @@ def test_group_sizes_and_ragged_tiles(nolo, n, bf16):
     run_both(nolo, W, n, 5 * 1024 + 3, 7, 3, dt, stride=5 * 1024 + 16)
 
 
+@pytest.mark.parametrize("n", [5, 6, 7, 9, 16, 17, 24, 32, 33, 48, 49, 64, 65, 96, 97, 100, 128, 129, 256, 300, 512, 520])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_large_subgroups(nolo, n, bf16):
+    """8 < n <= 512 runs the kernel that splits members across warps and, above 64 members,
+    across a thread-block cluster (with masked member slots when n does not fill them);
+    n > 512 the two-pass kernel.  Two subgroups, ragged P."""
+    dt = torch.bfloat16 if bf16 else torch.float32
+    run_both(nolo, 2 * n, n, 1000 + 3, 11, 4, dt)
+    if n in (16, 100, 128):
+        run_both(nolo, n, n, 257, 2, 9, dt, hp=(F[0], F[1], 0.0))     # one group of all workers
+
+
 @pytest.mark.parametrize("P", [1, 2, 3, 4, 5, 7, 8, 9, 1023, 1024, 1025, 2047, 2049, 4100])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_small_and_odd_P(nolo, P, bf16):
