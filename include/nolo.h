@@ -51,6 +51,7 @@ extern "C" {
 
 #define NOLO_KERNEL_OUTER 0 /* kernel ids for nolo_timing_read() */
 #define NOLO_KERNEL_ROUTE 1
+#define NOLO_KERNEL_DIVERGENCE 2
 
 typedef struct nolo_handle nolo_handle;
 
@@ -214,12 +215,28 @@ int nolo_get_groups(nolo_handle* h, int32_t* host_out);
 int nolo_get_route(nolo_handle* h, int32_t* host_out);
 
 /*
+ * Replica divergence of the bound slow weights phi: how far the W workers have
+ * drifted apart (the quantity plotted in Fig. 3b, the standard deviation of the
+ * model weights across the data-parallel replicas, before the figure's
+ * normalisation by the run's maximum).  For every parameter p the population
+ * variance var_p of phi[0..W-1][p] across the workers is formed; then
+ *   host_out[0] = (1/P) sum_p sqrt(var_p)      mean per-parameter standard deviation
+ *   host_out[1] = sqrt((1/P) sum_p var_p)      root of the mean variance
+ * (the paper does not say which of the two scalars it plots).  Read-only on
+ * phi; float32 per parameter, float64 sums in a fixed order (reproducible).
+ * Allocates 16 bytes per 2048 parameters of device scratch on first use.
+ * Synchronous: returns when the two doubles are in host memory.
+ * Errors: NOLO_EINVAL, NOLO_ESTATE, NOLO_ENOMEM, NOLO_ECUDA.
+ */
+int nolo_divergence(nolo_handle* h, double* host_out);
+
+/*
  * Device-time instrumentation.  With enable != 0 every later launch of the
- * fused outer-step kernel and of the routing copy kernel is bracketed by CUDA
+ * fused outer-step kernel, the routing copy kernel and the divergence kernels is bracketed by CUDA
  * events on the bound stream (up to 4096 launches per kernel between reads).
  * nolo_timing_read synchronises the stream, returns the summed device time in
  * milliseconds and the number of bracketed launches of `kernel`
- * (NOLO_KERNEL_OUTER / NOLO_KERNEL_ROUTE) since the last read, and resets them.
+ * (NOLO_KERNEL_OUTER / NOLO_KERNEL_ROUTE / NOLO_KERNEL_DIVERGENCE) since the last read, and resets them.
  */
 int nolo_timing_enable(nolo_handle* h, int enable);
 int nolo_timing_read(nolo_handle* h, int kernel, double* total_ms, int64_t* launches);

@@ -12,6 +12,9 @@ values, closed forms and invariants):
                          momentum over a subgroup of n workers) and Eq. 3
                          (slow-weight update), then the reset of the fast
                          weights to the new slow weights (Section 3.2).
+* ``divergence``      -- the replica spread plotted in Fig. 3b (standard
+                         deviation of the weights across the data-parallel
+                         replicas).
 * ``route_forward`` / ``route_backward`` -- Section 3.1 and Algorithm 1: every
                          step each stage boundary gets a fresh random
                          permutation of the replicas; activations follow it
@@ -203,6 +206,26 @@ def outer_step_seeded(phi, theta, delta, seed, step, n, alpha, beta, gamma,
     perm = draw_groups(seed, step, phi.shape[0], n)
     out = outer_step(phi, theta, delta, perm, n, alpha, beta, gamma, theta_dtype)
     return out + (perm,)
+
+
+# --------------------------------------------------------------------------
+# Replica divergence (Fig. 3b)
+# --------------------------------------------------------------------------
+
+def divergence(phi):
+    """Spread of the slow weights across the W data-parallel replicas (the
+    quantity of Fig. 3b, before its normalisation by the run's maximum).
+
+    For every parameter p: mean_p = (1/W) sum_w phi[w, p] and the population
+    variance var_p = (1/W) sum_w (phi[w, p] - mean_p)^2.  Returns
+    (mean_p sqrt(var_p), sqrt(mean_p var_p)); the paper does not say which
+    scalar it plots, so both are given.
+    """
+    x = np.asarray(phi).astype(np.float64)
+    W = x.shape[0]
+    mean = x.sum(axis=0) / W
+    var = ((x - mean) ** 2).sum(axis=0) / W
+    return float(np.sqrt(var).sum() / var.size), float(np.sqrt(var.sum() / var.size))
 
 
 # --------------------------------------------------------------------------

@@ -21,7 +21,7 @@ LIB_PATH = os.environ.get("NOLO_LIBRARY") or os.path.join(_HERE, "libnolo.so")
 
 NOLO_OK, NOLO_EINVAL, NOLO_ESTATE, NOLO_EALIGN, NOLO_ECUDA, NOLO_ENOMEM = 0, -1, -2, -3, -4, -5
 NOLO_F32, NOLO_BF16 = 0, 1
-NOLO_KERNEL_OUTER, NOLO_KERNEL_ROUTE = 0, 1
+NOLO_KERNEL_OUTER, NOLO_KERNEL_ROUTE, NOLO_KERNEL_DIVERGENCE = 0, 1, 2
 NOLO_MAX_WORKERS = 4096
 NOLO_STATIC_MAX_WORKERS = 1024
 
@@ -59,6 +59,7 @@ SIGNATURES = {
     "nolo_route_host": [_H, _u64, _u64, _vp, _vp, _vp],
     "nolo_get_groups": [_H, _vp],
     "nolo_get_route": [_H, _vp],
+    "nolo_divergence": [_H, ctypes.POINTER(ctypes.c_double)],
     "nolo_timing_enable": [_H, _i32],
     "nolo_timing_read": [_H, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)],
     "nolo_launch_count": [_H, ctypes.POINTER(_i64)],
@@ -202,6 +203,13 @@ def nolo_get_route(h: Handle) -> np.ndarray:
     out = np.empty((max(h.stages - 1, 0), h.K, h.W), dtype=np.int32)
     _check(_lib.nolo_get_route(h.ptr, out.ctypes.data), "nolo_get_route", h)
     return out
+
+
+def nolo_divergence(h: Handle):
+    """(mean per-parameter std across workers, root of the mean variance) of the bound phi."""
+    out = (ctypes.c_double * 2)()
+    _check(_lib.nolo_divergence(h.ptr, out), "nolo_divergence", h)
+    return out[0], out[1]
 
 
 def nolo_timing_enable(h: Handle, enable: bool = True):

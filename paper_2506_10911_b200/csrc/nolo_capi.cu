@@ -12,6 +12,7 @@
 namespace {
 
 constexpr int kMaxTimed = 4096;
+constexpr int kTimedKernels = 3;
 
 struct KernelTimer {
     cudaEvent_t* start = nullptr;
@@ -48,12 +49,16 @@ struct nolo_handle {
     int32_t* d_route = nullptr;  // [stages-1][K][W], owned
     bool route_valid = false;
 
+    // divergence metric scratch (allocated on first use)
+    void* d_div_partials = nullptr;
+    double* d_div_out = nullptr;
+
     // host-streaming helpers (created on first use)
     cudaStream_t s_in = nullptr, s_out = nullptr;
     cudaEvent_t ev_in = nullptr, ev_kernel = nullptr, ev_fence = nullptr;
 
     bool timing = false;
-    KernelTimer timers[2];
+    KernelTimer timers[kTimedKernels];
     int64_t launches = 0;
     char err[256] = {0};
 };
@@ -366,6 +371,28 @@ int nolo_get_route(nolo_handle* h, int32_t* host_out) {
     return NOLO_OK;
 }
 
+int nolo_divergence(nolo_handle* h, double* host_out) {
+    if (!h) return NOLO_EINVAL;
+    if (!host_out) return fail(h, NOLO_EINVAL, "host_out must not be NULL");
+    if (!h->state_bound) return fail(h, NOLO_ESTATE, "nolo_bind_state has not been called");
+    if (!h->d_div_partials) {
+        cudaError_t e = cudaMalloc(&h->d_div_partials, (size_t)nolo::divergence_partials(h->P) * 16);
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->d_div_out), 2 * sizeof(double));
+        if (e != cudaSuccess) {
+            if (h->d_div_partials) { cudaFree(h->d_div_partials); h->d_div_partials = nullptr; }
+            return fail(h, e == cudaErrorMemoryAllocation ? NOLO_ENOMEM : NOLO_ECUDA,
+                        "divergence scratch allocation: %s", cudaGetErrorString(e));
+        }
+    }
+    Bracket br(h, NOLO_KERNEL_DIVERGENCE);
+    NOLO_CUDA(h, nolo::launch_divergence(h->phi, h->W, h->stride, h->P, h->d_div_partials, h->d_div_out, h->stream));
+    br.done();
+    h->launches += 2;
+    NOLO_CUDA(h, cudaMemcpyAsync(host_out, h->d_div_out, 2 * sizeof(double), cudaMemcpyDeviceToHost, h->stream));
+    NOLO_CUDA(h, cudaStreamSynchronize(h->stream));
+    return NOLO_OK;
+}
+
 int nolo_timing_enable(nolo_handle* h, int enable) {
     if (!h) return NOLO_EINVAL;
     h->timing = enable != 0;
@@ -374,7 +401,7 @@ int nolo_timing_enable(nolo_handle* h, int enable) {
 
 int nolo_timing_read(nolo_handle* h, int kernel, double* total_ms, int64_t* launches) {
     if (!h) return NOLO_EINVAL;
-    if (kernel != NOLO_KERNEL_OUTER && kernel != NOLO_KERNEL_ROUTE)
+    if (kernel < 0 || kernel >= kTimedKernels)
         return fail(h, NOLO_EINVAL, "unknown kernel id %d", kernel);
     if (!total_ms || !launches) return fail(h, NOLO_EINVAL, "output pointers must not be NULL");
     NOLO_CUDA(h, cudaStreamSynchronize(h->stream));
@@ -412,6 +439,8 @@ int nolo_destroy(nolo_handle* h) {
     }
     if (h->d_perm) cudaFree(h->d_perm);
     if (h->d_route) cudaFree(h->d_route);
+    if (h->d_div_partials) cudaFree(h->d_div_partials);
+    if (h->d_div_out) cudaFree(h->d_div_out);
     delete h;
     return NOLO_OK;
 }

@@ -45,4 +45,11 @@ struct RouteArgs {
 
 cudaError_t launch_route(const RouteArgs& a, cudaStream_t stream);
 
+// Replica divergence of phi (Fig. 3b): out2[0] = mean over parameters of the across-worker
+// population standard deviation, out2[1] = sqrt(mean over parameters of the across-worker variance).
+// `partials` is device scratch of divergence_partials(P) * 16 bytes; out2 is device memory.
+int64_t divergence_partials(int64_t P);
+cudaError_t launch_divergence(const float* phi, int W, int64_t stride, int64_t P, void* partials,
+                              double* out2, cudaStream_t stream);
+
 }  // namespace nolo

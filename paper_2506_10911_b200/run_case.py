@@ -35,6 +35,7 @@ def main(argv=None):
     ap.add_argument("--M", type=int, default=0, help="micro-batches per boundary (0: no routing)")
     ap.add_argument("--E", type=int, default=0, help="elements per micro-batch activation")
     ap.add_argument("--act", choices=["f32", "bf16"], default="bf16")
+    ap.add_argument("--divergence", action="store_true", help="also time the replica-divergence metric")
     ap.add_argument("--fast-fill", action="store_true", help="fill state with one uniform pass instead of the "
                     "per-chunk normal/drift recipe (timing only; values do not affect the kernels' time)")
     args = ap.parse_args(argv)
@@ -95,6 +96,12 @@ def main(argv=None):
            "outer_ms": ms / max(cnt, 1), "bytes_per_param": bpp,
            "outer_gbs": bpp * args.W * P / (ms / max(cnt, 1) * 1e-3) / 1e9,
            "params_per_s": args.W * P / (ms / max(cnt, 1) * 1e-3)}
+    if args.divergence:
+        for _ in range(args.steps):
+            nolo.nolo_divergence(h)
+        dms, dcnt = nolo.nolo_timing_read(h, nolo.NOLO_KERNEL_DIVERGENCE)
+        res.update(divergence_ms=dms / max(dcnt, 1),
+                   divergence_gbs=4 * args.W * P / (dms / max(dcnt, 1) * 1e-3) / 1e9)
     if route:
         rms, rcnt = nolo.nolo_timing_read(h, nolo.NOLO_KERNEL_ROUTE)
         rbytes = 2 * acts.numel() * acts.element_size()

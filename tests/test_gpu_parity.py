@@ -271,6 +271,37 @@ def test_route_host_path(nolo):
     nolo.nolo_destroy(h)
 
 
+# --------------------------------------------------------------- divergence
+
+@pytest.mark.parametrize("W,P", [(1, 10), (2, 4099), (8, 1 << 16), (16, 300_001), (128, 5000), (1000, 513)])
+def test_divergence_matches_oracle(nolo, W, P):
+    phi, theta, delta = synth.make_state(W, P, 4, pad_value=float("nan"))
+    phi[:, :P] = phi[:1, :P] + 0.05 * phi[:, :P]            # replicas close to a common point
+    dev = [x.cuda() for x in (phi, theta, delta)]
+    h = nolo.nolo_create(W, 1, P, 1, *F)
+    nolo.nolo_bind_state(h, *dev)
+    got = nolo.nolo_divergence(h)
+    want = O.divergence(to_np(phi)[:, :P])
+    assert got[0] == pytest.approx(want[0], rel=1e-5, abs=1e-12)
+    assert got[1] == pytest.approx(want[1], rel=1e-5, abs=1e-12)
+    assert nolo.nolo_divergence(h) == got                    # reproducible bit for bit
+    assert torch.equal(dev[0].cpu().view(torch.int32), phi.view(torch.int32))     # read-only
+    nolo.nolo_destroy(h)
+
+
+def test_divergence_after_gossip_step_is_zero(nolo):
+    """alpha = beta = 0, gamma = 1, n = W puts every replica on the mean."""
+    W, P = 16, 70_000
+    dev = [x.cuda() for x in synth.make_state(W, P, 6)]
+    h = nolo.nolo_create(W, W, P, 1, 0.0, 0.0, 1.0)
+    nolo.nolo_bind_state(h, *dev)
+    before = nolo.nolo_divergence(h)
+    nolo.nolo_outer_step(h, 0, 0)
+    after = nolo.nolo_divergence(h)
+    assert before[0] > 1e-2 and after[1] < 1e-8
+    nolo.nolo_destroy(h)
+
+
 # ----------------------------------------------------- boundary behaviour
 
 def test_error_codes(nolo):

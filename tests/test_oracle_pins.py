@@ -348,6 +348,60 @@ def test_noisy_quadratic_converges_to_neighbourhood():
     assert 1.5 < var[0.2] / var[0.1] < 4.5
 
 
+# ------------------------------------------------------------ divergence
+
+def test_divergence_closed_forms():
+    # hand example: values 1,2,3,4 across 4 workers: mean 2.5, population variance 1.25
+    a, b = O.divergence(np.array([[1.0], [2.0], [3.0], [4.0]], dtype=F32))
+    assert abs(a - 1.25 ** 0.5) < 1e-12 and abs(b - 1.25 ** 0.5) < 1e-12
+    # two workers: std = |x0 - x1| / 2 per parameter
+    x = np.array([[1.0, -2.0, 0.5], [3.0, -2.0, 0.0]], dtype=F32)
+    a, b = O.divergence(x)
+    assert abs(a - (1.0 + 0.0 + 0.25) / 3) < 1e-12
+    assert abs(b - ((1.0 + 0.0 + 0.0625) / 3) ** 0.5) < 1e-12
+    # identical replicas have no spread; one worker has none either
+    assert O.divergence(np.tile(x[0], (5, 1))) == (0.0, 0.0)
+    assert O.divergence(x[:1]) == (0.0, 0.0)
+
+
+def test_divergence_against_numpy_and_invariances():
+    rng = np.random.default_rng(3)
+    x = (0.02 * rng.normal(size=(9, 1001)) + rng.normal(size=(1, 1001))).astype(F32)
+    a, b = O.divergence(x)
+    sd = np.std(x.astype(np.float64), axis=0)              # library routine, ddof = 0
+    assert abs(a - sd.mean()) < 1e-14 and abs(b - np.sqrt((sd ** 2).mean())) < 1e-14
+    assert a <= b + 1e-15                                   # Jensen: mean of roots <= root of mean
+    sh = O.divergence((x.astype(np.float64) + 7.0))
+    assert abs(sh[0] - a) < 1e-12 and abs(sh[1] - b) < 1e-12
+    sc = O.divergence(x.astype(np.float64) * -3.0)
+    assert abs(sc[0] - 3 * a) < 1e-12 and abs(sc[1] - 3 * b) < 1e-12
+    assert O.divergence(x[rng.permutation(9)]) == pytest.approx((a, b), rel=1e-14)
+    # brute force with python floats on a tiny case
+    t = x[:3, :4].astype(np.float64)
+    tot_s = tot_v = 0.0
+    for p in range(4):
+        m = sum(t[w, p] for w in range(3)) / 3
+        v = sum((t[w, p] - m) ** 2 for w in range(3)) / 3
+        tot_s += v ** 0.5
+        tot_v += v
+    got = O.divergence(x[:3, :4])
+    assert abs(got[0] - tot_s / 4) < 1e-15 and abs(got[1] - (tot_v / 4) ** 0.5) < 1e-15
+
+
+def test_gossip_step_removes_divergence_and_pull_shrinks_it():
+    """Spread identity: with alpha = 0 a full-group step scales the spread by (1 - gamma)."""
+    W, P = 8, 500
+    phi, theta, delta = rnd_state(W, P, 12)
+    perm = np.arange(W, dtype=np.int32)
+    before = O.divergence(phi)
+    p1, _, _ = O.outer_step(phi, theta, delta, perm, W, 0.0, 0.7, 0.25)
+    after = O.divergence(p1)
+    assert after[0] == pytest.approx(0.75 * before[0], rel=1e-5)
+    assert after[1] == pytest.approx(0.75 * before[1], rel=1e-5)
+    p2, _, _ = O.outer_step(phi, theta, delta, perm, W, 0.0, 0.7, 1.0)
+    assert O.divergence(p2)[1] < 1e-8 * before[1] + 1e-9
+
+
 # ------------------------------------------------------------------ routing
 
 def test_route_tables_are_permutations():
