@@ -7,30 +7,11 @@
 // indices in ascending (key, index) order.  Integer arithmetic only, so the tables are
 // reproducible bit for bit on any machine.
 #include "nolo_internal.h"
+#include "nolo_philox.cuh"
 
 namespace nolo {
 
 namespace {
-
-// Published Philox4x64 multipliers and Weyl key increments.
-constexpr uint64_t kM0 = 0xD2E7470EE14C6C93ull;
-constexpr uint64_t kM1 = 0xCA5A826395121157ull;
-constexpr uint64_t kW0 = 0x9E3779B97F4A7C15ull;
-constexpr uint64_t kW1 = 0xBB67AE8584CAA73Bull;
-
-__device__ __forceinline__ uint64_t philox4x64_10_word0(uint64_t c0, uint64_t c1, uint64_t c2,
-                                                        uint64_t c3, uint64_t k0, uint64_t k1) {
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-        const uint64_t hi0 = __umul64hi(kM0, c0), lo0 = kM0 * c0;
-        const uint64_t hi1 = __umul64hi(kM1, c2), lo1 = kM1 * c2;
-        const uint64_t n0 = hi1 ^ c1 ^ k0;
-        const uint64_t n2 = hi0 ^ c3 ^ k1;
-        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
-        k0 += kW0; k1 += kW1;
-    }
-    return c0;
-}
 
 constexpr int kDrawThreads = 256;
 
@@ -44,7 +25,7 @@ draw_perm_kernel(uint64_t seed, uint64_t step, uint64_t domain, int N, int slots
     const int b = blockIdx.x / slots_drawn;
     const int s = blockIdx.x % slots_drawn;
     for (int i = threadIdx.x; i < N; i += blockDim.x)
-        keys[i] = philox4x64_10_word0((uint64_t)i, (uint64_t)b, (uint64_t)s, domain, seed, step);
+        keys[i] = draw_key((uint64_t)i, (uint64_t)b, (uint64_t)s, domain, seed, step);
     __syncthreads();
     const int k_lo = (slots_drawn == slots_total) ? s : 0;
     const int k_hi = (slots_drawn == slots_total) ? s + 1 : slots_total;
