@@ -231,6 +231,56 @@ int nolo_get_route(nolo_handle* h, int32_t* host_out);
 int nolo_divergence(nolo_handle* h, double* host_out);
 
 /*
+ * Monte-Carlo estimate of the completion time of a binary-tree all-reduce
+ * over W workers when every message takes an independent LogNormal(mu,
+ * sigma^2) time (Section 4.3 and the latency-analysis appendix; Fig. 5a): a
+ * parent is ready when both children's messages have arrived, the result then
+ * descends the same tree, and the all-reduce ends when the last leaf has it.
+ * With constant message time t_c this is the paper's 2 t_c log2(W); with W = 2
+ * it is the pair exchange of local averaging, max(t1,t2) + max(t3,t4).
+ *   W       power of two, 2..NOLO_MAX_WORKERS;  sigma >= 0;  trials 1..2^24
+ *   seed    random stream: the message on the edge above heap node c (2..2W-1)
+ *           in phase p (0 up, 1 down) of trial s uses philox4x64-10(counter =
+ *           (c, s, p, 3), key = (seed, 0)); u = ((word >> 11) + 0.5) 2^-53;
+ *           z = sqrt(-2 ln u(word0)) cos(2 pi u(word1)); t = exp(mu + sigma z)
+ *   stream  cudaStream_t for the kernels
+ *   host_stats   host, 2 doubles: mean completion time, its standard error
+ *   host_trials  host, [trials] completion times, or NULL
+ * float64 arithmetic.  Synchronous; allocates and frees its own scratch.
+ * Errors: NOLO_EINVAL, NOLO_ENOMEM, NOLO_ECUDA.
+ */
+int nolo_sim_tree_allreduce(int W, double mu, double sigma, int64_t trials, uint64_t seed,
+                            void* stream, double* host_stats, double* host_trials);
+
+/*
+ * Expected time of the pair exchange, E[max(t1,t2) + max(t3,t4)] =
+ * 2 (1 + erf(sigma/2)) exp(mu + sigma^2/2) for i.i.d. LogNormal(mu, sigma^2)
+ * message times (the appendix's closed form): the denominator of Fig. 5a's
+ * ratio.  Host arithmetic only.
+ */
+double nolo_expected_pair_exchange(double mu, double sigma);
+
+/*
+ * Monte-Carlo simulation of the cost of the global barrier (Section 4.3,
+ * Fig. 5b): every inner step of every worker takes an independent
+ * LogNormal(mu, sigma^2) time (the paper: mu = 1, sigma^2 = 0.5), communication
+ * is free.  Under DiLoCo all W workers meet after every H inner steps; under
+ * NoLoCo a worker only waits for the n members of its random subgroup (the
+ * same draw as nolo_outer_step, with step = outer iteration and boundary =
+ * trial).  Reports the time for all workers to finish T outer iterations.
+ *   seed    inner step k of worker w in outer iteration t of trial s uses
+ *           philox4x64-10(counter = (k, w, t, 4), key = (seed, s)), transformed
+ *           as in nolo_sim_tree_allreduce
+ *   host_stats   host, 4 doubles: mean time with the global barrier, mean time
+ *           with subgroup waits, then the standard errors of the two means
+ *   host_trials  host, [trials][2] (barrier, subgroup) per trial, or NULL
+ * Synchronous; allocates and frees its own scratch.  trials 1..2^20.
+ * Errors: NOLO_EINVAL, NOLO_ENOMEM, NOLO_ECUDA.
+ */
+int nolo_sim_straggler(int W, int n, int H, int T, double mu, double sigma, int64_t trials,
+                       uint64_t seed, void* stream, double* host_stats, double* host_trials);
+
+/*
  * Device-time instrumentation.  With enable != 0 every later launch of the
  * fused outer-step kernel, the routing copy kernel and the divergence kernels is bracketed by CUDA
  * events on the bound stream (up to 4096 launches per kernel between reads).

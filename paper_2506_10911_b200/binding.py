@@ -60,6 +60,9 @@ SIGNATURES = {
     "nolo_get_groups": [_H, _vp],
     "nolo_get_route": [_H, _vp],
     "nolo_divergence": [_H, ctypes.POINTER(ctypes.c_double)],
+    "nolo_sim_tree_allreduce": [_i32, ctypes.c_double, ctypes.c_double, _i64, _u64, _vp, _vp, _vp],
+    "nolo_expected_pair_exchange": [ctypes.c_double, ctypes.c_double],
+    "nolo_sim_straggler": [_i32, _i32, _i32, _i32, ctypes.c_double, ctypes.c_double, _i64, _u64, _vp, _vp, _vp],
     "nolo_timing_enable": [_H, _i32],
     "nolo_timing_read": [_H, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)],
     "nolo_launch_count": [_H, ctypes.POINTER(_i64)],
@@ -71,7 +74,8 @@ SIGNATURES = {
 for _name, _args in SIGNATURES.items():
     _fn = getattr(_lib, _name)
     _fn.argtypes = _args
-    _fn.restype = ctypes.c_char_p if _name in ("nolo_strerror", "nolo_last_error") else ctypes.c_int
+    _fn.restype = (ctypes.c_char_p if _name in ("nolo_strerror", "nolo_last_error")
+                   else ctypes.c_double if _name == "nolo_expected_pair_exchange" else ctypes.c_int)
 
 
 def _ptr(x) -> int:
@@ -210,6 +214,37 @@ def nolo_divergence(h: Handle):
     out = (ctypes.c_double * 2)()
     _check(_lib.nolo_divergence(h.ptr, out), "nolo_divergence", h)
     return out[0], out[1]
+
+
+def _stream_ptr(stream):
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def nolo_sim_tree_allreduce(W: int, mu: float, sigma: float, trials: int, seed: int, stream=None,
+                            return_trials: bool = False):
+    """Returns (mean completion time, standard error[, per-trial times])."""
+    stats = np.empty(2, dtype=np.float64)
+    per = np.empty(trials, dtype=np.float64) if return_trials else None
+    _check(_lib.nolo_sim_tree_allreduce(W, mu, sigma, trials, seed, _stream_ptr(stream), stats.ctypes.data,
+                                        per.ctypes.data if return_trials else None), "nolo_sim_tree_allreduce")
+    return (stats[0], stats[1], per) if return_trials else (stats[0], stats[1])
+
+
+def nolo_expected_pair_exchange(mu: float, sigma: float) -> float:
+    return _lib.nolo_expected_pair_exchange(mu, sigma)
+
+
+def nolo_sim_straggler(W: int, n: int, H: int, T: int, mu: float, sigma: float, trials: int, seed: int,
+                       stream=None, return_trials: bool = False):
+    """Returns (mean barrier time, mean subgroup time, their standard errors[, per-trial [trials, 2]])."""
+    stats = np.empty(4, dtype=np.float64)
+    per = np.empty((trials, 2), dtype=np.float64) if return_trials else None
+    _check(_lib.nolo_sim_straggler(W, n, H, T, mu, sigma, trials, seed, _stream_ptr(stream), stats.ctypes.data,
+                                   per.ctypes.data if return_trials else None), "nolo_sim_straggler")
+    return tuple(stats) + ((per,) if return_trials else ())
 
 
 def nolo_timing_enable(h: Handle, enable: bool = True):

@@ -445,6 +445,46 @@ int nolo_destroy(nolo_handle* h) {
     return NOLO_OK;
 }
 
+int nolo_sim_tree_allreduce(int W, double mu, double sigma, int64_t trials, uint64_t seed, void* stream,
+                            double* host_stats, double* host_trials) {
+    if (W < 2 || W > NOLO_MAX_WORKERS || (W & (W - 1)) || trials < 1 || trials > (int64_t(1) << 24) ||
+        !std::isfinite(mu) || !std::isfinite(sigma) || sigma < 0 || !host_stats)
+        return NOLO_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    double* d = nullptr;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&d), sizeof(double) * ((size_t)trials + 4));
+    if (e != cudaSuccess) return e == cudaErrorMemoryAllocation ? NOLO_ENOMEM : NOLO_ECUDA;
+    e = nolo::launch_tree_allreduce(W, mu, sigma, trials, seed, d + 4, d, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(host_stats, d, 2 * sizeof(double), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && host_trials)
+        e = cudaMemcpyAsync(host_trials, d + 4, sizeof(double) * (size_t)trials, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    cudaFree(d);
+    return e == cudaSuccess ? NOLO_OK : NOLO_ECUDA;
+}
+
+int nolo_sim_straggler(int W, int n, int H, int T, double mu, double sigma, int64_t trials, uint64_t seed,
+                       void* stream, double* host_stats, double* host_trials) {
+    if (W < 1 || W > NOLO_MAX_WORKERS || n < 1 || n > W || W % n != 0 || H < 1 || T < 1 || trials < 1 ||
+        trials > (int64_t(1) << 20) || !std::isfinite(mu) || !std::isfinite(sigma) || sigma < 0 || !host_stats)
+        return NOLO_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    double* d = nullptr;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&d), sizeof(double) * (2 * (size_t)trials + 4));
+    if (e != cudaSuccess) return e == cudaErrorMemoryAllocation ? NOLO_ENOMEM : NOLO_ECUDA;
+    e = nolo::launch_straggler(W, n, H, T, mu, sigma, trials, seed, d + 4, d, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(host_stats, d, 4 * sizeof(double), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && host_trials)
+        e = cudaMemcpyAsync(host_trials, d + 4, sizeof(double) * 2 * (size_t)trials, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    cudaFree(d);
+    return e == cudaSuccess ? NOLO_OK : NOLO_ECUDA;
+}
+
+double nolo_expected_pair_exchange(double mu, double sigma) {
+    return 2.0 * (1.0 + std::erf(sigma / 2.0)) * std::exp(mu + sigma * sigma / 2.0);
+}
+
 const char* nolo_strerror(int status) {
     switch (status) {
         case NOLO_OK: return "ok";

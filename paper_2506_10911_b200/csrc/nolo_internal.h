@@ -52,4 +52,11 @@ int64_t divergence_partials(int64_t P);
 cudaError_t launch_divergence(const float* phi, int W, int64_t stride, int64_t P, void* partials,
                               double* out2, cudaStream_t stream);
 
+// Latency simulations (Section 4.3).  per_trial: device [trials] resp. [trials][2];
+// stats: device, the column means followed by their standard errors.
+cudaError_t launch_tree_allreduce(int W, double mu, double sigma, int64_t trials, uint64_t seed,
+                                  double* per_trial, double* stats, cudaStream_t stream);
+cudaError_t launch_straggler(int W, int n, int H, int T, double mu, double sigma, int64_t trials,
+                             uint64_t seed, double* per_trial, double* stats, cudaStream_t stream);
+
 }  // namespace nolo
