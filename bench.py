@@ -133,24 +133,31 @@ class ClockSampler:
 # ----------------------------------------------------------------------------
 
 def oracle_sample_state(cols: int, seed: int = 0):
+    """The first `cols` columns of the workload's state and the matching share of its routed
+    activations, as numpy arrays (bfloat16 as uint16 bit patterns)."""
+    wl = workload()
     phi, theta, delta = synth.make_state(W, cols, seed, torch.bfloat16)
-    return [x.view(torch.int16).numpy().view(np.uint16) if x.dtype == torch.bfloat16 else x.numpy()
-            for x in (phi, theta, delta)]
+    e_s = max(1, int(wl["E"] * cols / wl["P"]))
+    acts = synth.make_acts(STAGES - 1, W, wl["M"] // W, e_s, 1000 + seed, torch.bfloat16)
+    as_np = lambda x: x.view(torch.int16).numpy().view(np.uint16) if x.dtype == torch.bfloat16 else x.numpy()  # noqa: E731
+    return [as_np(x) for x in (phi, theta, delta, acts)]
 
 
 def time_oracle_step(state, k: int) -> float:
+    """One step of the oracle as it stands: outer step, then routing."""
     from oracle import nolo_oracle as O
     t0 = time.perf_counter()
     O.outer_step_seeded(state[0], state[1], state[2], k, k, N_GROUP, ALPHA, BETA, GAMMA, O.THETA_BF16)
+    O.route_forward(state[3], O.draw_route(k, k, STAGES, W, state[3].shape[2]))
     return time.perf_counter() - t0
 
 
-def cpu_baseline(cols: int = 1 << 22):
-    """One oracle outer step on the first `cols` columns x all W rows."""
+def cpu_baseline(cols: int = 1 << 24):
+    """One oracle step on the first `cols` columns x all W rows."""
     state = oracle_sample_state(cols)
     dt = time_oracle_step(state, 0)
     return {"value": W * cols / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"1 outer step on {cols} of {workload()['P']} columns x {W} workers "
+            "sample": f"1 step (outer step + routing) on {cols} of {workload()['P']} columns x {W} workers "
                       f"(numpy float64, single thread), {dt:.1f} s"}
 
 
@@ -171,7 +178,8 @@ def run_reference(args):
         time_oracle_step(state, k)
     dt = time.perf_counter() - t0
     value = W * cols * args.steps / dt
-    sample = f"each step = 1 oracle outer step on {cols} of {wl['P']} columns x {W} workers (numpy float64, 1 thread)"
+    sample = (f"each step = 1 oracle step (outer step + routing) on {cols} of {wl['P']} columns x {W} workers "
+              f"(numpy float64, 1 thread)")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
@@ -323,7 +331,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-cols", type=int, default=1 << 22)
+    ap.add_argument("--cpu-cols", type=int, default=1 << 24)
     args = ap.parse_args()
     args.warmup = max(3, args.warmup)
     if args.impl == "reference":

@@ -224,7 +224,7 @@ int nolo_get_route(nolo_handle* h, int32_t* host_out);
  *   host_out[1] = sqrt((1/P) sum_p var_p)      root of the mean variance
  * (the paper does not say which of the two scalars it plots).  Read-only on
  * phi; float32 per parameter, float64 sums in a fixed order (reproducible).
- * Allocates 16 bytes per 2048 parameters of device scratch on first use.
+ * Allocates 16 bytes per 4096 parameters of device scratch on first use.
  * Synchronous: returns when the two doubles are in host memory.
  * Errors: NOLO_EINVAL, NOLO_ESTATE, NOLO_ENOMEM, NOLO_ECUDA.
  */

@@ -12,8 +12,15 @@ namespace nolo {
 
 namespace {
 
+#ifndef NOLO_DIV_ITEMS
+#define NOLO_DIV_ITEMS 4
+#endif
+#ifndef NOLO_DIV_UNROLL
+#define NOLO_DIV_UNROLL 4
+#endif
 constexpr int kThreads = 256;
-constexpr int kItems = 2;       // quads per thread
+constexpr int kItems = NOLO_DIV_ITEMS;       // quads per thread
+constexpr int kUnroll = NOLO_DIV_UNROLL;    // worker rows in flight per thread
 
 struct Welford4 {
     float4 mean, m2;
@@ -44,7 +51,7 @@ divergence_partial_kernel(const float* __restrict__ phi, int W, int64_t stride, 
     bool ok[kItems];
 #pragma unroll
     for (int it = 0; it < kItems; ++it) ok[it] = q0 + (int64_t)it * kThreads < full_quads;
-#pragma unroll 4
+#pragma unroll kUnroll
     for (int w = 0; w < W; ++w) {
         const float4* row = reinterpret_cast<const float4*>(phi + (int64_t)w * stride);
         const float inv_k = __frcp_rn((float)(w + 1));
