@@ -258,10 +258,31 @@ def run_ours(args):
     job_ms, job_units = replicas.job_time_and_units(local_ms, float(W) * P * args.steps, dev)
     value = replicas.throughput(job_units, job_ms)
 
+    # ---- a plain copy of our own in the same run, as context for the roofline fraction
+    copy_gbs = None
+    if rank == 0:
+        try:
+            nbytes = 4 << 30
+            src = torch.empty(nbytes, dtype=torch.uint8, device=dev).fill_(1)
+            dst = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+            copy_gbs = nolo.nolo_copy_probe(src, dst, nbytes, 10)
+            del src, dst
+        except Exception:
+            copy_gbs = None
+
     # ---- end to end: state and activations in pinned host memory, through the host entry points
     e2e = None
     e2e_note = None
-    if not args.no_e2e:
+    host_need = world * (W * stride * 10 + 2 * acts.numel() * acts.element_size())
+    try:
+        import psutil
+        host_free = psutil.virtual_memory().available
+    except Exception:
+        host_free = None
+    if not args.no_e2e and host_free is not None and host_need > 0.5 * host_free:
+        e2e_note = (f"skipped: page-locking {host_need / 1e9:.0f} GB for {world} replicas would take more than "
+                    f"half of the {host_free / 1e9:.0f} GB of free host memory")
+    elif not args.no_e2e:
         try:
             h_state = [torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for x in (phi, theta, delta)]
             for hs, ds in zip(h_state, (phi, theta, delta)):
@@ -316,7 +337,8 @@ def run_ours(args):
                      "traffic": PROFILED_DRAM_BYTES_PER_PARAM * W * P,
                      "traffic_note": "ncu dram bytes of a 1.34 GB case of this kernel scaled by columns",
                      "bytes_per_launch": BYTES_PER_PARAM * W * P,
-                     "ms_per_launch": per_launch_ms, "launches_timed": outer_cnt},
+                     "ms_per_launch": per_launch_ms, "launches_timed": outer_cnt,
+                     "plain_copy_same_run_gbs": copy_gbs},
         "route": {"ms_per_launch": route_ms / max(1, route_cnt), "bytes_per_launch": route_bytes,
                   "achieved_gbs": route_bytes / (route_ms / max(1, route_cnt) * 1e-3) / 1e9 if route_ms else None},
     }

@@ -281,6 +281,20 @@ int nolo_sim_straggler(int W, int n, int H, int T, double mu, double sigma, int6
                        uint64_t seed, void* stream, double* host_stats, double* host_trials);
 
 /*
+ * (Measurement aid; the paper has no counterpart.)  Times a plain
+ * device-to-device copy of `bytes` bytes with the routing kernel's access
+ * pattern (one-shot grid, 128-bit streaming loads and stores): 3 warm-up
+ * copies, then `iters` copies between CUDA events on `stream`.  The bandwidth
+ * 2 * bytes / time is the practical HBM ceiling for a half-read, half-write
+ * kernel on this device, against which the other kernels can be read.
+ *   src, dst  device, 16-byte aligned, disjoint;  bytes a positive multiple of 16
+ *   ms_per_copy  host, receives the mean milliseconds per copy
+ * Synchronous.  Errors: NOLO_EINVAL, NOLO_EALIGN, NOLO_ECUDA.
+ */
+int nolo_copy_probe(const void* src, void* dst, int64_t bytes, int iters, void* stream,
+                    double* ms_per_copy);
+
+/*
  * Device-time instrumentation.  With enable != 0 every later launch of the
  * fused outer-step kernel, the routing copy kernel and the divergence kernels is bracketed by CUDA
  * events on the bound stream (up to 4096 launches per kernel between reads).

@@ -2,7 +2,7 @@
 simulated speed-up", and the latency-analysis appendix).
 
 THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT: plain NumPy float64, used only
-to judge the CUDA simulation kernels.  Shares no code with them.
+to check the CUDA simulation kernels.  Shares no code with them.
 
 Two simulations, as the paper describes them:
 

@@ -1,7 +1,7 @@
 """CPU oracle for the NoLoCo outer synchronisation step and random pipeline routing.
 
 THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a plain, slow, float64
-restatement of the method, written from the paper, used only to judge the CUDA
+restatement of the method, written from the paper, used only to check the CUDA
 path (tests, the smoke check and the benchmark's CPU-baseline leg).  It shares
 no code with the CUDA library and imports nothing from it.
 

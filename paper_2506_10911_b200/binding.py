@@ -60,6 +60,7 @@ SIGNATURES = {
     "nolo_get_groups": [_H, _vp],
     "nolo_get_route": [_H, _vp],
     "nolo_divergence": [_H, ctypes.POINTER(ctypes.c_double)],
+    "nolo_copy_probe": [_vp, _vp, _i64, _i32, _vp, ctypes.POINTER(ctypes.c_double)],
     "nolo_sim_tree_allreduce": [_i32, ctypes.c_double, ctypes.c_double, _i64, _u64, _vp, _vp, _vp],
     "nolo_expected_pair_exchange": [ctypes.c_double, ctypes.c_double],
     "nolo_sim_straggler": [_i32, _i32, _i32, _i32, ctypes.c_double, ctypes.c_double, _i64, _u64, _vp, _vp, _vp],
@@ -221,6 +222,14 @@ def _stream_ptr(stream):
     if stream is None:
         stream = torch.cuda.current_stream()
     return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def nolo_copy_probe(src, dst, nbytes: int, iters: int = 10, stream=None) -> float:
+    """GB/s (read + write bytes) of a plain copy of nbytes from src to dst."""
+    ms = ctypes.c_double()
+    _check(_lib.nolo_copy_probe(_ptr(src), _ptr(dst), nbytes, iters, _stream_ptr(stream), ctypes.byref(ms)),
+           "nolo_copy_probe")
+    return 2.0 * nbytes / (ms.value * 1e-3) / 1e9
 
 
 def nolo_sim_tree_allreduce(W: int, mu: float, sigma: float, trials: int, seed: int, stream=None,

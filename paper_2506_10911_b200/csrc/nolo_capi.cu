@@ -445,6 +445,28 @@ int nolo_destroy(nolo_handle* h) {
     return NOLO_OK;
 }
 
+int nolo_copy_probe(const void* src, void* dst, int64_t bytes, int iters, void* stream, double* ms_per_copy) {
+    if (!src || !dst || bytes < 16 || bytes % 16 != 0 || iters < 1 || !ms_per_copy) return NOLO_EINVAL;
+    if (!aligned16(src) || !aligned16(dst)) return NOLO_EALIGN;
+    if (overlap(src, (size_t)bytes, dst, (size_t)bytes)) return NOLO_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaEvent_t a = nullptr, b = nullptr;
+    cudaError_t e = cudaEventCreate(&a);
+    if (e == cudaSuccess) e = cudaEventCreate(&b);
+    for (int i = 0; e == cudaSuccess && i < 3; ++i) e = nolo::launch_copy_probe(src, dst, bytes, s);   // warm-up
+    if (e == cudaSuccess) e = cudaEventRecord(a, s);
+    for (int i = 0; e == cudaSuccess && i < iters; ++i) e = nolo::launch_copy_probe(src, dst, bytes, s);
+    if (e == cudaSuccess) e = cudaEventRecord(b, s);
+    if (e == cudaSuccess) e = cudaEventSynchronize(b);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, a, b);
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    if (e != cudaSuccess) return NOLO_ECUDA;
+    *ms_per_copy = (double)ms / iters;
+    return NOLO_OK;
+}
+
 int nolo_sim_tree_allreduce(int W, double mu, double sigma, int64_t trials, uint64_t seed, void* stream,
                             double* host_stats, double* host_trials) {
     if (W < 2 || W > NOLO_MAX_WORKERS || (W & (W - 1)) || trials < 1 || trials > (int64_t(1) << 24) ||

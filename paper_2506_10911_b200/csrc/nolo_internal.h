@@ -45,6 +45,9 @@ struct RouteArgs {
 
 cudaError_t launch_route(const RouteArgs& a, cudaStream_t stream);
 
+// Plain copy of `bytes` (a multiple of 16) with the routing kernel's access pattern.
+cudaError_t launch_copy_probe(const void* in, void* out, int64_t bytes, cudaStream_t stream);
+
 // Replica divergence of phi (Fig. 3b): out2[0] = mean over parameters of the across-worker
 // population standard deviation, out2[1] = sqrt(mean over parameters of the across-worker variance).
 // `partials` is device scratch of divergence_partials(P) * 16 bytes; out2 is device memory.

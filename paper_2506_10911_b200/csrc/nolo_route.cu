@@ -79,6 +79,24 @@ route_copy_elem_kernel(const T* __restrict__ in, T* __restrict__ out, const int3
     }
 }
 
+// Plain device-to-device copy with the same access pattern as the routing copy (one tile of
+// 256 x kVecPerThread 128-bit vectors per CTA): the yardstick the other kernels are compared with.
+__global__ void __launch_bounds__(kThreads)
+copy_probe_kernel(const uint4* __restrict__ in, uint4* __restrict__ out, int64_t vecs) {
+    const int64_t v0 = (int64_t)blockIdx.x * kTileVecs + threadIdx.x;
+    uint4 v[kVecPerThread];
+#pragma unroll
+    for (int i = 0; i < kVecPerThread; ++i) {
+        const int64_t x = v0 + (int64_t)i * kThreads;
+        if (x < vecs) v[i] = __ldcs(in + x);
+    }
+#pragma unroll
+    for (int i = 0; i < kVecPerThread; ++i) {
+        const int64_t x = v0 + (int64_t)i * kThreads;
+        if (x < vecs) __stcs(out + x, v[i]);
+    }
+}
+
 // One CTA per tile (a one-shot grid streams through memory in address order, which measured
 // about 10 % faster on B200 than a resident grid striding over the tiles); the kernels still loop
 // so that a tile count beyond the grid limit stays correct.
@@ -87,6 +105,16 @@ int tile_grid(int64_t total_tiles) {
 }
 
 }  // namespace
+
+cudaError_t launch_copy_probe(const void* in, void* out, int64_t bytes, cudaStream_t stream) {
+    const int64_t vecs = bytes / 16;
+    const int64_t tiles = (vecs + kTileVecs - 1) / kTileVecs;
+    if (tiles <= 0) return cudaSuccess;
+    if (tiles > 0x7fffffffll) return cudaErrorInvalidConfiguration;
+    copy_probe_kernel<<<(unsigned)tiles, kThreads, 0, stream>>>(static_cast<const uint4*>(in),
+                                                                static_cast<uint4*>(out), vecs);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_route(const RouteArgs& a, cudaStream_t stream) {
     const int64_t blocks = (int64_t)a.B * a.R * a.K;

@@ -365,6 +365,19 @@ def test_timing_and_launch_count(nolo):
     nolo.nolo_destroy(h)
 
 
+def test_copy_probe(nolo):
+    src = torch.arange(1 << 22, dtype=torch.int32, device="cuda")
+    dst = torch.zeros_like(src)
+    gbs = nolo.nolo_copy_probe(src, dst, src.numel() * 4, 3)
+    assert torch.equal(src, dst) and gbs > 10
+    with pytest.raises(nolo.NoloError) as e:
+        nolo.nolo_copy_probe(src, src, src.numel() * 4, 3)
+    assert e.value.status == nolo.NOLO_EINVAL
+    with pytest.raises(nolo.NoloError) as e:
+        nolo.nolo_copy_probe(src, dst, 24, 3)
+    assert e.value.status == nolo.NOLO_EINVAL
+
+
 def test_non_default_stream(nolo):
     W, n, P = 4, 2, 10_000
     phi, theta, delta = synth.make_state(W, P, 2)
