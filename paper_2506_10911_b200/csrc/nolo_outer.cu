@@ -235,8 +235,8 @@ struct SplitShape {
 template <int MPW, typename ThetaT, bool CLUSTER, int MAXW>
 __global__ void __launch_bounds__(MAXW * 32, SplitShape<MPW, MAXW>::kMinBlocks)
 outer_step_split_kernel(const KArgs a, int members_per_cta) {
-    __shared__ float4 part_D[kSplitMaxWarps][32];
-    __shared__ float4 part_P[kSplitMaxWarps][32];
+    __shared__ float4 part_D[MAXW][32];
+    __shared__ float4 part_P[MAXW][32];
     __shared__ float4 cta_D[32];
     __shared__ float4 cta_P[32];
     const int G = blockDim.x >> 5;

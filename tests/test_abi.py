@@ -78,3 +78,13 @@ def test_null_handle_is_an_error_not_a_crash(lib):
     assert raw.nolo_destroy(None) == lib.NOLO_OK
     raw.nolo_create.argtypes = lib.SIGNATURES["nolo_create"]
     assert raw.nolo_create(4, 2, 8, 1, 0.5, 0.7, 0.5, None) == lib.NOLO_EINVAL
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    """There is no fallback path: without the shared library the binding cannot be imported."""
+    import subprocess
+    import sys
+    env = dict(os.environ, NOLO_LIBRARY=str(tmp_path / "absent.so"))
+    res = subprocess.run([sys.executable, "-c", "from paper_2506_10911_b200 import binding"], cwd=ROOT, env=env,
+                         capture_output=True, text=True)
+    assert res.returncode != 0 and "ImportError" in res.stderr and "no CPU or PyTorch fallback" in res.stderr
