@@ -5,6 +5,8 @@ memory from cudaMalloc, so it must give exactly what nolo_outer_step gives.
 Checked on two calls in a row, of different shapes, because the table is
 shared between calls and keeps the previous call's contents."""
 
+import gc
+
 import pytest
 import torch
 
@@ -38,10 +40,11 @@ def test_static_entry_point_matches_handle_path_twice(nolo):
         state = synth.make_state(W, P, seed, dt)
         want = reference_step(nolo, W, n, P, state, seed, step)
         dev = [x.clone().cuda() for x in state]
+        gc.collect()                                     # leftovers of earlier tests may be freed at any time
         before = torch.cuda.memory_allocated()
         nolo.nolo_outer_step_static(W, n, P, *HP, *dev, seed, step)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == before
+        assert torch.cuda.memory_allocated() <= before   # the call itself took nothing from torch's pool
         for got, w in zip(dev, want):
             # same kernels, same table: identical bits (tighter than the 2e-6 / 1e-7 parity tolerance)
             assert torch.equal(got, w)
