@@ -180,6 +180,20 @@ int nolo_bind_route(nolo_handle* h, int M, int64_t E, int act_dtype,
 int nolo_route(nolo_handle* h, uint64_t seed, uint64_t step, const void* acts);
 
 /*
+ * Forward routing of ONE stage boundary (what a single stage of Algorithm 1
+ * does when it receives its inputs): draws table[boundary][:][:] for
+ * (seed, step) -- the same permutation nolo_route would draw for that
+ * boundary -- and gathers
+ *   out_b[r][k][:] = acts_b[table[boundary][k][r]][k][:].
+ *   boundary  0 .. stages-2
+ *   acts_b, out_b  device, [W][K][E] of that boundary, 16-byte aligned, disjoint
+ * Rows of the table that belong to other boundaries keep whatever an earlier
+ * call left there.  Asynchronous.  Errors: as nolo_route.
+ */
+int nolo_route_boundary(nolo_handle* h, uint64_t seed, uint64_t step, int boundary,
+                        const void* acts_b, void* out_b);
+
+/*
  * Backward routing (Algorithm 1, backward pass: gradients return along the
  * path of the forward pass): with the table of (seed, step),
  *   grads_out[b][table[b][k][r]][k][:] = grads[b][r][k][:].

@@ -55,6 +55,7 @@ SIGNATURES = {
     "nolo_outer_step_host": [_H, _u64, _u64, _vp, _vp, _vp, _i64],
     "nolo_bind_route": [_H, _i32, _i64, _i32, _vp, _i32],
     "nolo_route": [_H, _u64, _u64, _vp],
+    "nolo_route_boundary": [_H, _u64, _u64, _i32, _vp, _vp],
     "nolo_route_backward": [_H, _u64, _u64, _vp, _vp],
     "nolo_route_host": [_H, _u64, _u64, _vp, _vp, _vp],
     "nolo_get_groups": [_H, _vp],
@@ -187,6 +188,11 @@ def nolo_bind_route(h: Handle, M: int, E: int, acts_out, per_microbatch: bool = 
 
 def nolo_route(h: Handle, seed: int, step: int, acts):
     _check(_lib.nolo_route(h.ptr, seed, step, _ptr(acts)), "nolo_route", h)
+
+
+def nolo_route_boundary(h: Handle, seed: int, step: int, boundary: int, acts_b, out_b):
+    _check(_lib.nolo_route_boundary(h.ptr, seed, step, boundary, _ptr(acts_b), _ptr(out_b)),
+           "nolo_route_boundary", h)
 
 
 def nolo_route_backward(h: Handle, seed: int, step: int, grads, grads_out):

@@ -324,6 +324,34 @@ int nolo_route(nolo_handle* h, uint64_t seed, uint64_t step, const void* acts) {
     return enqueue_route(h, seed, step, acts, h->acts_out, 0);
 }
 
+int nolo_route_boundary(nolo_handle* h, uint64_t seed, uint64_t step, int boundary, const void* acts_b,
+                        void* out_b) {
+    if (!h) return NOLO_EINVAL;
+    if (!h->route_bound) return fail(h, NOLO_ESTATE, "nolo_bind_route has not been called");
+    if (boundary < 0 || boundary >= h->stages - 1)
+        return fail(h, NOLO_EINVAL, "boundary %d is outside 0..%d", boundary, h->stages - 2);
+    if (!acts_b || !out_b) return fail(h, NOLO_EINVAL, "acts_b and out_b must not be NULL");
+    if (!aligned16(acts_b) || !aligned16(out_b)) return fail(h, NOLO_EALIGN, "pointers must be 16-byte aligned");
+    const size_t bytes = route_bytes(h) / (size_t)(h->stages - 1);
+    if (overlap(acts_b, bytes, out_b, bytes)) return fail(h, NOLO_EINVAL, "acts_b overlaps out_b");
+    const int drawn = h->per_microbatch ? h->K : 1;
+    NOLO_CUDA(h, nolo::launch_draw_range(seed, step, nolo::kDomainRoute, h->W, boundary, 1, drawn, h->K,
+                                         h->d_route, h->stream));
+    ++h->launches;
+    h->route_valid = true;
+    nolo::RouteArgs a;
+    a.in = acts_b; a.out = out_b;
+    a.table = h->d_route + (size_t)boundary * h->K * h->W;
+    a.B = 1; a.R = h->W; a.K = h->K; a.E = h->E;
+    a.elem_size = elem_size(h->act_dtype);
+    a.backward = 0;
+    Bracket br(h, NOLO_KERNEL_ROUTE);
+    NOLO_CUDA(h, nolo::launch_route(a, h->stream));
+    br.done();
+    ++h->launches;
+    return NOLO_OK;
+}
+
 int nolo_route_backward(nolo_handle* h, uint64_t seed, uint64_t step, const void* grads, void* grads_out) {
     if (!h) return NOLO_EINVAL;
     if (!h->route_bound) return fail(h, NOLO_ESTATE, "nolo_bind_route has not been called");

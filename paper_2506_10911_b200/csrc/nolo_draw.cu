@@ -19,10 +19,10 @@ constexpr int kDrawThreads = 256;
 // elements that sort before it (rank by counting: N <= 4096, so N^2 compares are cheap and need
 // no sort network).
 __global__ void __launch_bounds__(kDrawThreads)
-draw_perm_kernel(uint64_t seed, uint64_t step, uint64_t domain, int N, int slots_drawn,
+draw_perm_kernel(uint64_t seed, uint64_t step, uint64_t domain, int N, int first_boundary, int slots_drawn,
                  int slots_total, int32_t* __restrict__ table) {
     extern __shared__ uint64_t keys[];
-    const int b = blockIdx.x / slots_drawn;
+    const int b = first_boundary + blockIdx.x / slots_drawn;
     const int s = blockIdx.x % slots_drawn;
     for (int i = threadIdx.x; i < N; i += blockDim.x)
         keys[i] = draw_key((uint64_t)i, (uint64_t)b, (uint64_t)s, domain, seed, step);
@@ -43,13 +43,19 @@ draw_perm_kernel(uint64_t seed, uint64_t step, uint64_t domain, int N, int slots
 
 }  // namespace
 
-cudaError_t launch_draw(uint64_t seed, uint64_t step, int domain, int N, int boundaries,
-                        int slots_drawn, int slots_total, int32_t* table, cudaStream_t stream) {
+cudaError_t launch_draw_range(uint64_t seed, uint64_t step, int domain, int N, int first_boundary,
+                              int boundaries, int slots_drawn, int slots_total, int32_t* table,
+                              cudaStream_t stream) {
     const int blocks = boundaries * slots_drawn;
     if (blocks <= 0 || N <= 0) return cudaSuccess;
     draw_perm_kernel<<<blocks, kDrawThreads, (size_t)N * sizeof(uint64_t), stream>>>(
-        seed, step, (uint64_t)domain, N, slots_drawn, slots_total, table);
+        seed, step, (uint64_t)domain, N, first_boundary, slots_drawn, slots_total, table);
     return cudaGetLastError();
+}
+
+cudaError_t launch_draw(uint64_t seed, uint64_t step, int domain, int N, int boundaries,
+                        int slots_drawn, int slots_total, int32_t* table, cudaStream_t stream) {
+    return launch_draw_range(seed, step, domain, N, 0, boundaries, slots_drawn, slots_total, table, stream);
 }
 
 }  // namespace nolo

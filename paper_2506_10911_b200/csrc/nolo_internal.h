@@ -17,6 +17,12 @@ constexpr int kDomainRoute = 2;   // counter word 3 for routing draws
 cudaError_t launch_draw(uint64_t seed, uint64_t step, int domain, int N, int boundaries,
                         int slots_drawn, int slots_total, int32_t* table, cudaStream_t stream);
 
+// The same for boundaries first_boundary .. first_boundary + boundaries - 1 only (table indexed by the
+// absolute boundary).
+cudaError_t launch_draw_range(uint64_t seed, uint64_t step, int domain, int N, int first_boundary,
+                              int boundaries, int slots_drawn, int slots_total, int32_t* table,
+                              cudaStream_t stream);
+
 struct OuterArgs {
     float* phi;          // [W][stride]
     void* theta;         // [W][stride] float or bf16

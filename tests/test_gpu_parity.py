@@ -247,6 +247,27 @@ def test_route_bit_exact(nolo, S, R, K, E, dt, pm):
     nolo.nolo_destroy(h)
 
 
+@pytest.mark.parametrize("pm", [False, True])
+def test_route_one_boundary_at_a_time(nolo, pm):
+    S, R, K, E = 4, 8, 2, 3000
+    acts = synth.make_acts(S - 1, R, K, E, 5, torch.bfloat16)
+    d_acts = acts.cuda()
+    d_out = torch.zeros_like(d_acts)
+    h = nolo.nolo_create(R, 2, 8, S, *F)
+    nolo.nolo_bind_route(h, R * K, E, torch.zeros_like(d_acts), pm)
+    table = O.draw_route(6, 2, S, R, K, pm)
+    want = O.route_forward(to_np(acts), table)
+    for b in (2, 0, 1):
+        nolo.nolo_route_boundary(h, 6, 2, b, d_acts[b], d_out[b])
+        torch.cuda.synchronize()
+        assert np.array_equal(to_np(d_out[b]), want[b])
+    assert np.array_equal(nolo.nolo_get_route(h), table)
+    with pytest.raises(nolo.NoloError) as e:
+        nolo.nolo_route_boundary(h, 6, 2, 3, d_acts[0], d_out[0])
+    assert e.value.status == nolo.NOLO_EINVAL
+    nolo.nolo_destroy(h)
+
+
 def test_route_single_stage_is_a_noop(nolo):
     h = nolo.nolo_create(4, 2, 8, 1, *F)
     out = torch.zeros(8, device="cuda")
