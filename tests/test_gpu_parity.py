@@ -120,6 +120,34 @@ def test_heavy_tailed_drift(nolo):
     run_both(nolo, 32, 8, 1 << 14, 3, 1, drift="student_t3")
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+def test_nan_and_inf_propagate_within_their_subgroup_only(nolo, bf16):
+    """No special-casing: a NaN or Inf in one member's column poisons that column for the members
+    of its subgroup and nothing else."""
+    W, n, P = 8, 2, 2048 + 5
+    dt = torch.bfloat16 if bf16 else torch.float32
+    phi, theta, delta = synth.make_state(W, P, 13, dt)
+    phi[3, 17] = float("nan")
+    theta[5, 100] = float("inf")
+    delta[0, 2050] = float("-inf")            # in the ragged tail
+    d = [x.cuda() for x in (phi, theta, delta)]
+    h = nolo.nolo_create(W, n, P, 1, *F)
+    nolo.nolo_bind_state(h, *d)
+    nolo.nolo_outer_step(h, 2, 2)
+    torch.cuda.synchronize()
+    perm = nolo.nolo_get_groups(h)
+    nolo.nolo_destroy(h)
+    want = O.outer_step(to_np(phi)[:, :P], to_np(theta)[:, :P], to_np(delta)[:, :P], perm, n, *F,
+                        O.THETA_BF16 if bf16 else O.THETA_F32)
+    got_phi = to_np(d[0])[:, :P]
+    assert np.array_equal(np.isfinite(got_phi), np.isfinite(want[0]))
+    assert np.array_equal(np.isnan(got_phi), np.isnan(want[0]))
+    bad = ~np.isfinite(want[0])
+    assert 3 <= bad.sum() <= 5                  # 2 members x 2 columns, plus the one row with -inf momentum
+    assert_close_f32(np.where(bad, 0, got_phi), np.where(bad, 0, want[0]), "phi")
+    assert np.array_equal(got_phi[bad & ~np.isnan(want[0])], want[0][bad & ~np.isnan(want[0])])   # signed Inf
+
+
 def test_diloco_reduction_on_gpu(nolo):
     """n = W, gamma = 0, shared momentum: all replicas take the same global
     momentum step on the mean outer gradient (Section 3.2)."""
