@@ -45,9 +45,9 @@ MICROBATCH_TOKENS = 4 * 1024    # 4 sequences of 1024 tokens per micro-batch
 BYTES_PER_PARAM = 20            # read phi4+theta2+delta4, write phi4+delta4+theta2
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per worker-parameter of the fused kernel, from the profiler's dram__bytes_read.sum +
-# dram__bytes_write.sum on a 1.34 GB case of the same kernel (W=16, n=2, bf16 theta, P=2^23: 2.6269 GB
+# dram__bytes_write.sum on a 1.34 GB case of the same kernel (W=16, n=2, bf16 theta, P=2^23: 2.6283 GB
 # for 134 217 728 worker-parameters); traffic is proportional to the columns processed.
-PROFILED_DRAM_BYTES_PER_PARAM = 2.6269e9 / (16 * 8388608)
+PROFILED_DRAM_BYTES_PER_PARAM = 2.6283e9 / (16 * 8388608)
 
 
 def workload():
@@ -332,7 +332,7 @@ def run_ours(args):
         "clocks": clocks,
         "e2e": e2e if e2e is not None else {"value": None, "unit": UNIT, "note": e2e_note or "skipped"},
         "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "kernel": "outer_step_reg_kernel<2,bf16>", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "outer_step_reg_kernel<2,bf16,1>", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "traffic": PROFILED_DRAM_BYTES_PER_PARAM * W * P,
                      "traffic_note": "ncu dram bytes of a 1.34 GB case of this kernel scaled by columns",
