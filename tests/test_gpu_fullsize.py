@@ -97,6 +97,50 @@ def test_config2_125M_bf16_ten_steps(nolo):
     run_config(nolo, 16, 2, synth.model_params("125M"), torch.bfloat16, (F32(.5), F32(.7), F32(.5)), steps=10)
 
 
+def test_config2_every_element_by_sum_and_difference_identities(nolo):
+    """Full coverage at full size without a host copy.  For a pair (n = 2), Eq. 2-3 fix the sum and
+    the difference of the two members' new slow weights:
+        phi_a' + phi_b' = (phi_a + phi_b) + alpha (delta_a + delta_b) - beta (Delta_a + Delta_b)
+        phi_a' - phi_b' = (1 - gamma) (phi_a - phi_b) + alpha (delta_a - delta_b)
+    and the two together fix every element.  Checked on the device in float64 for all 2e9 elements
+    of the 125M x 16 configuration, with delta' = phi' - phi and theta' = round(phi')."""
+    W, n, P = 16, 2, synth.model_params("125M")
+    a_, b_, c_ = F32(.5), F32(.7), F32(.5)
+    stride = synth.padded_stride(P)
+    need_gb(2 * W * stride * 10 / 1e9 + 12)
+    dev = torch.device("cuda")
+    phi = torch.empty((W, stride), dtype=torch.float32, device=dev)
+    theta = torch.empty((W, stride), dtype=torch.bfloat16, device=dev)
+    delta = torch.empty((W, stride), dtype=torch.float32, device=dev)
+    synth.fill_state_(phi, theta, delta, P, seed=3)
+    phi0, theta0, delta0 = phi.clone(), theta.clone(), delta.clone()
+    h = nolo.nolo_create(W, n, P, 1, a_, b_, c_)
+    nolo.nolo_bind_state(h, phi, theta, delta)
+    nolo.nolo_outer_step(h, 3, 0)
+    torch.cuda.synchronize()
+    perm = O.draw_groups(3, 0, W, n)
+    assert np.array_equal(nolo.nolo_get_groups(h), perm)
+    nolo.nolo_destroy(h)
+    chunk = 1 << 24
+    for g in range(W // n):
+        a, b = int(perm[2 * g]), int(perm[2 * g + 1])
+        for c0 in range(0, P, chunk):
+            sl = slice(c0, min(P, c0 + chunk))
+            pa, pb = phi0[a, sl].double(), phi0[b, sl].double()
+            da, db = delta0[a, sl].double(), delta0[b, sl].double()
+            Da, Db = pa - theta0[a, sl].double(), pb - theta0[b, sl].double()
+            na, nb = phi[a, sl].double(), phi[b, sl].double()
+            want_sum = (pa + pb) + a_ * (da + db) - b_ * (Da + Db)
+            want_dif = (1 - c_) * (pa - pb) + a_ * (da - db)
+            tol = 2 * (1e-7 + 2e-6 * torch.maximum(pa.abs(), pb.abs()))
+            assert bool(((na + nb - want_sum).abs() <= tol).all()), f"sum identity, group {g}"
+            assert bool(((na - nb - want_dif).abs() <= tol).all()), f"difference identity, group {g}"
+            for r, p0, pn in ((a, pa, na), (b, pb, nb)):
+                d_new = delta[r, sl].double()
+                assert bool(((d_new - (pn - p0)).abs() <= 1e-7 + 2e-6 * d_new.abs()).all()), "delta' != phi' - phi"
+                assert torch.equal(phi[r, sl].to(torch.bfloat16), theta[r, sl])
+
+
 @pytest.mark.parametrize("gamma", [0.0, 0.5])
 def test_config3_1p3B_fp32_three_steps(nolo, gamma):
     """W=8, n=4, 1.3B decoder, all fp32 (about 126 GB resident)."""
