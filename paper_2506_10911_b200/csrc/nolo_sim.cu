@@ -16,6 +16,10 @@ namespace nolo {
 
 namespace {
 
+#ifndef NOLO_TREE_THREADS
+#define NOLO_TREE_THREADS 128
+#endif
+constexpr int kTreeThreads = NOLO_TREE_THREADS;   // small CTAs: the upper tree levels leave few threads busy
 constexpr uint64_t kDomainTree = 3;
 constexpr uint64_t kDomainStraggler = 4;
 
@@ -170,7 +174,7 @@ cudaError_t launch_tree_allreduce(int W, double mu, double sigma, int64_t trials
     cudaError_t e = cudaFuncSetAttribute(tree_allreduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem);
     if (e != cudaSuccess) return e;
-    tree_allreduce_kernel<<<(unsigned)trials, round_up_threads(W / 2), smem, stream>>>(W, mu, sigma, seed,
+    tree_allreduce_kernel<<<(unsigned)trials, round_up_threads(W / 2 < kTreeThreads ? W / 2 : kTreeThreads), smem, stream>>>(W, mu, sigma, seed,
                                                                                         per_trial);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
