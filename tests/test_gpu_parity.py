@@ -148,6 +148,33 @@ def test_nan_and_inf_propagate_within_their_subgroup_only(nolo, bf16):
     assert np.array_equal(got_phi[bad & ~np.isnan(want[0])], want[0][bad & ~np.isnan(want[0])])   # signed Inf
 
 
+@pytest.mark.parametrize("W,n", [(4, 2), (8, 8), (24, 12), (72, 72), (130, 130), (600, 600)])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_guard_bands_around_every_buffer_stay_intact(nolo, W, n, bf16):
+    """Each state tensor sits between two 4 KiB bands of a known pattern inside a larger
+    allocation; no kernel path (register-resident, warp-split, cluster, two-pass, ragged tail)
+    may write outside its rows."""
+    P, stride, band = 1000 + 3, 1008, 1024            # band in elements
+    dt = torch.bfloat16 if bf16 else torch.float32
+    state = synth.make_state(W, P, 8, dt, stride=stride, pad_value=7.0)
+    bufs, views = [], []
+    for x in state:
+        big = torch.full((2 * band + W * stride,), -123.0, dtype=x.dtype, device="cuda")
+        v = big[band:band + W * stride].view(W, stride)
+        v.copy_(x)
+        bufs.append(big)
+        views.append(v)
+    h = nolo.nolo_create(W, n, P, 1, *F)
+    nolo.nolo_bind_state(h, *views)
+    nolo.nolo_outer_step(h, 1, 1)
+    torch.cuda.synchronize()
+    nolo.nolo_destroy(h)
+    for big, v in zip(bufs, views):
+        assert bool((big[:band] == -123.0).all()) and bool((big[-band:] == -123.0).all()), "guard band written"
+        assert bool((v[:, P:] == 7.0).all()), "padding written"
+    assert not torch.equal(views[0][:, :P].cpu(), state[0][:, :P])       # and the step did run
+
+
 def test_diloco_reduction_on_gpu(nolo):
     """n = W, gamma = 0, shared momentum: all replicas take the same global
     momentum step on the mean outer gradient (Section 3.2)."""
