@@ -324,6 +324,26 @@ def test_route_one_boundary_at_a_time(nolo, pm):
     nolo.nolo_destroy(h)
 
 
+@pytest.mark.parametrize("E,dt", [(4096 + 8, torch.bfloat16), (1001, torch.bfloat16), (333, torch.float32)])
+def test_route_guard_bands(nolo, E, dt):
+    S, R, K, band = 3, 4, 2, 2048
+    acts = synth.make_acts(S - 1, R, K, E, 4, dt).cuda()
+    n_el = acts.numel()
+    big = torch.full((2 * band + n_el,), -5.0, dtype=dt, device="cuda")
+    out = big[band:band + n_el].view_as(acts)
+    h = nolo.nolo_create(R, 2, 8, S, *F)
+    nolo.nolo_bind_route(h, R * K, E, out)
+    nolo.nolo_route(h, 1, 2, acts)
+    big2 = torch.full((2 * band + n_el,), -5.0, dtype=dt, device="cuda")
+    back = big2[band:band + n_el].view_as(acts)
+    nolo.nolo_route_backward(h, 1, 2, out, back)
+    torch.cuda.synchronize()
+    nolo.nolo_destroy(h)
+    for b in (big, big2):
+        assert bool((b[:band] == -5.0).all()) and bool((b[-band:] == -5.0).all())
+    assert torch.equal(back, acts)
+
+
 def test_route_single_stage_is_a_noop(nolo):
     h = nolo.nolo_create(4, 2, 8, 1, *F)
     out = torch.zeros(8, device="cuda")
