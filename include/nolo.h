@@ -309,6 +309,17 @@ int nolo_copy_probe(const void* src, void* dst, int64_t bytes, int iters, void* 
                     double* ms_per_copy);
 
 /*
+ * Device-side status of this handle's kernels.  The outer-step kernel for
+ * subgroups of 65 to 192 members waits on a shared-memory barrier for its
+ * bulk copies; that wait is bounded, and a CTA whose wait ever ran out leaves
+ * its tile of the state untouched and raises this word instead of hanging.
+ *   host_out  receives 0 (nothing happened) or 1 (a wait ran out since the
+ *             handle was created: the last outer steps are incomplete)
+ * Synchronises the stream.  Errors: NOLO_EINVAL, NOLO_ECUDA.
+ */
+int nolo_device_status(nolo_handle* h, int32_t* host_out);
+
+/*
  * Device-time instrumentation.  With enable != 0 every later launch of the
  * fused outer-step kernel, the routing copy kernel and the divergence kernels is bracketed by CUDA
  * events on the bound stream (up to 4096 launches per kernel between reads).

@@ -65,6 +65,7 @@ SIGNATURES = {
     "nolo_sim_tree_allreduce": [_i32, ctypes.c_double, ctypes.c_double, _i64, _u64, _vp, _vp, _vp],
     "nolo_expected_pair_exchange": [ctypes.c_double, ctypes.c_double],
     "nolo_sim_straggler": [_i32, _i32, _i32, _i32, ctypes.c_double, ctypes.c_double, _i64, _u64, _vp, _vp, _vp],
+    "nolo_device_status": [_H, ctypes.POINTER(ctypes.c_int32)],
     "nolo_timing_enable": [_H, _i32],
     "nolo_timing_read": [_H, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)],
     "nolo_launch_count": [_H, ctypes.POINTER(_i64)],
@@ -221,6 +222,12 @@ def nolo_divergence(h: Handle):
     out = (ctypes.c_double * 2)()
     _check(_lib.nolo_divergence(h.ptr, out), "nolo_divergence", h)
     return out[0], out[1]
+
+
+def nolo_device_status(h: Handle) -> int:
+    out = ctypes.c_int32(-1)
+    _check(_lib.nolo_device_status(h.ptr, ctypes.byref(out)), "nolo_device_status", h)
+    return out.value
 
 
 def _stream_ptr(stream):

@@ -39,6 +39,7 @@ struct nolo_handle {
     bool state_bound = false;
 
     int32_t* d_perm = nullptr;   // [W], owned
+    int32_t* d_status = nullptr; // 1 word, owned: raised by a kernel whose bounded wait ran out
     bool groups_valid = false;
 
     // routing
@@ -134,6 +135,7 @@ int enqueue_outer(nolo_handle* h, int64_t col0, int64_t cols) {
     a.n = h->n;
     a.theta_bf16 = h->theta_dtype == NOLO_BF16;
     a.alpha = h->alpha; a.beta = h->beta; a.gamma = h->gamma;
+    a.status = h->d_status;
     Bracket br(h, NOLO_KERNEL_OUTER);
     NOLO_CUDA(h, nolo::launch_outer(a, h->stream));
     br.done();
@@ -203,6 +205,8 @@ int nolo_create(int W, int n, int64_t P, int stages, float alpha, float beta, fl
     }
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaMalloc(&h->d_perm, sizeof(int32_t) * (size_t)W);
+    if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(int32_t));
     if (e != cudaSuccess) {
         const int code = (e == cudaErrorMemoryAllocation) ? NOLO_ENOMEM : NOLO_ECUDA;
         nolo_destroy(h);
@@ -421,6 +425,14 @@ int nolo_divergence(nolo_handle* h, double* host_out) {
     return NOLO_OK;
 }
 
+int nolo_device_status(nolo_handle* h, int32_t* host_out) {
+    if (!h) return NOLO_EINVAL;
+    if (!host_out) return fail(h, NOLO_EINVAL, "host_out must not be NULL");
+    NOLO_CUDA(h, cudaMemcpyAsync(host_out, h->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, h->stream));
+    NOLO_CUDA(h, cudaStreamSynchronize(h->stream));
+    return NOLO_OK;
+}
+
 int nolo_timing_enable(nolo_handle* h, int enable) {
     if (!h) return NOLO_EINVAL;
     h->timing = enable != 0;
@@ -466,6 +478,7 @@ int nolo_destroy(nolo_handle* h) {
         delete[] t.stop;
     }
     if (h->d_perm) cudaFree(h->d_perm);
+    if (h->d_status) cudaFree(h->d_status);
     if (h->d_route) cudaFree(h->d_route);
     if (h->d_div_partials) cudaFree(h->d_div_partials);
     if (h->d_div_out) cudaFree(h->d_div_out);

@@ -33,6 +33,7 @@ struct OuterArgs {
     int W, n;
     int theta_bf16;
     float alpha, beta, gamma;
+    int32_t* status = nullptr;  // device word set to 1 if a bounded wait in a kernel ever runs out; may be NULL
 };
 
 // Fused Eq. 1-3 + theta reset over columns [0, P) of the rows (pointers may be pre-offset by

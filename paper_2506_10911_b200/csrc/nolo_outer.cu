@@ -203,7 +203,7 @@ outer_step_reg_kernel(const KArgs a) {
     if ((a.P & 3) && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) scalar_tail<ThetaT>(a, g);
 }
 
-// ---- large subgroups (8 < n <= 512): members split across warps, CTAs and a cluster --------
+// ---- large subgroups (8 < n <= 64, 192 < n <= 512): members split across warps, CTAs and a cluster
 //
 // Holding phi of every member of a tile in registers costs n x 512 bytes per 32 quads, and the
 // kernel only streams at full bandwidth while more than one CTA fits on an SM (one CTA's loads
@@ -342,6 +342,162 @@ outer_step_split_kernel(const KArgs a, int members_per_cta) {
     if (CLUSTER) cg::this_cluster().barrier_wait();   // peers may still be reading this CTA's sums
 }
 
+// ---- 64 < n <= 192: phi staged in shared memory by bulk-async copies ------------------------
+//
+// One CTA of 8 warps (16 above 112 members) owns one subgroup x 32 quads, for all n members.  The members' phi segments
+// (512 bytes each) are brought into shared memory by cp.async.bulk copies that complete on one
+// mbarrier, so phi needs no registers while it waits for the reduction; meanwhile every warp
+// streams the theta segments of its own members through registers and sums them.  After the
+// mbarrier and one CTA barrier each warp updates its own members: phi from shared memory, delta
+// from global memory.  sum_Delta is formed as sum(phi) - sum(theta), both in a fixed order.
+// Still one read and one write per element; n x 512 bytes of shared memory per CTA, 3 CTAs per SM
+// at n = 128, 2 at n = 192.  Measured 2 to 19 % faster than spreading such a subgroup over a cluster
+// of CTAs; from about 256 members on the cluster kernel below is the faster one again.
+// The wait on the mbarrier is bounded: if it ever ran out, the CTA would leave its
+// tile untouched and raise the status word instead of hanging.
+#ifndef NOLO_STAGED
+#define NOLO_STAGED 1
+#endif
+#ifndef NOLO_STAGED_MAX_N
+#define NOLO_STAGED_MAX_N 192
+#endif
+#ifndef NOLO_STAGED_SPLIT
+#define NOLO_STAGED_SPLIT 112      // up to here 8 warps, above 16 (8 to 14 members per warp)
+#endif
+constexpr int kStagedChunk = 4;      // member rows in flight per thread
+constexpr int kStagedWaitLimit = 1 << 20;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+template <typename ThetaT, int kStagedWarps>
+__global__ void __launch_bounds__(kStagedWarps * 32, kStagedWarps <= 8 ? 3 : 2)
+outer_step_staged_kernel(const KArgs a, int32_t* __restrict__ status) {
+    extern __shared__ __align__(128) unsigned char staged_smem[];
+    float4* phi_s = reinterpret_cast<float4*>(staged_smem);          // [n][32] quads
+    __shared__ float4 part_T[kStagedWarps][32];
+    __shared__ float4 part_P[kStagedWarps][32];
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int timed_out;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = blockIdx.y;
+    const int n = a.n;
+    const int32_t* members = a.perm + (int64_t)g * n;
+    const int64_t full_quads = a.P >> 2;
+    const int64_t q0 = (int64_t)blockIdx.x * 32;
+    const int tile_quads = (int)(full_quads - q0 < 32 ? (full_quads - q0 > 0 ? full_quads - q0 : 0) : 32);
+    const uint32_t row_bytes = (uint32_t)tile_quads * 16u;
+    const uint32_t bar_addr = smem_u32(&bar);
+
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_addr) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        timed_out = 0;
+    }
+    __syncthreads();
+    if (warp == 0 && tile_quads > 0) {
+        if (lane == 0)
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr),
+                         "r"((uint32_t)n * row_bytes)
+                         : "memory");
+        __syncwarp();
+        for (int j = lane; j < n; j += 32) {
+            const float* src = a.phi + (int64_t)__ldg(members + j) * a.stride + q0 * 4;
+            asm volatile(
+                "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                    smem_u32(phi_s + (size_t)j * 32)),
+                "l"(src), "r"(row_bytes), "r"(bar_addr)
+                : "memory");
+        }
+    }
+
+    // theta of this warp's members, through registers
+    const int mpw = (n + kStagedWarps - 1) / kStagedWarps;
+    const int j_begin = warp * mpw;
+    const int j_end = min(n, j_begin + mpw);
+    const bool ok = lane < tile_quads;
+    const int64_t q = q0 + lane;
+    float4 sT = make_float4(0.f, 0.f, 0.f, 0.f), sP = sT;
+    if (ok) {
+        for (int j = j_begin; j < j_end; j += kStagedChunk) {
+            typename ThetaRaw<ThetaT>::type raw[kStagedChunk];
+#pragma unroll
+            for (int i = 0; i < kStagedChunk; ++i)
+                if (j + i < j_end)
+                    raw[i] = load_theta_raw(
+                        static_cast<const ThetaT*>(a.theta) + (int64_t)__ldg(members + j + i) * a.stride, q);
+#pragma unroll
+            for (int i = 0; i < kStagedChunk; ++i)
+                if (j + i < j_end) {
+                    const float4 t = widen(raw[i]);
+                    sT.x += t.x; sT.y += t.y; sT.z += t.z; sT.w += t.w;
+                }
+        }
+    }
+    if (tile_quads > 0) {                     // bounded wait for the phi segments
+        bool done = false;
+        for (int it = 0; it < kStagedWaitLimit && !done; ++it) {
+            uint32_t ready;
+            asm volatile(
+                "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n selp.u32 %0, 1, 0, p;\n}\n"
+                : "=r"(ready)
+                : "r"(bar_addr)
+                : "memory");
+            done = ready != 0;
+        }
+        if (!done) timed_out = 1;
+    }
+    if (ok && !timed_out) {
+        for (int j = j_begin; j < j_end; ++j) {
+            const float4 p = phi_s[(size_t)j * 32 + lane];
+            sP.x += p.x; sP.y += p.y; sP.z += p.z; sP.w += p.w;
+        }
+    }
+    part_T[warp][lane] = sT;
+    part_P[warp][lane] = sP;
+    __syncthreads();
+    if (timed_out) {                           // same value in every thread after the barrier
+        if (threadIdx.x == 0 && status) atomicExch(status, 1);
+        return;
+    }
+    if (ok) {
+        float4 tT = part_T[0][lane], tP = part_P[0][lane];
+#pragma unroll
+        for (int w = 1; w < kStagedWarps; ++w) {
+            const float4 t = part_T[w][lane], p = part_P[w][lane];
+            tT.x += t.x; tT.y += t.y; tT.z += t.z; tT.w += t.w;
+            tP.x += p.x; tP.y += p.y; tP.z += p.z; tP.w += p.w;
+        }
+        const float4 sD = make_float4(tP.x - tT.x, tP.y - tT.y, tP.z - tT.z, tP.w - tT.w);
+        const float4 mP = make_float4(tP.x * a.inv_n, tP.y * a.inv_n, tP.z * a.inv_n, tP.w * a.inv_n);
+        for (int j = j_begin; j < j_end; j += kStagedChunk) {
+            float4 dl[kStagedChunk];
+            int64_t off[kStagedChunk];
+#pragma unroll
+            for (int i = 0; i < kStagedChunk; ++i)
+                if (j + i < j_end) {
+                    off[i] = (int64_t)__ldg(members + j + i) * a.stride;
+                    dl[i] = __ldcs(reinterpret_cast<const float4*>(a.delta + off[i]) + q);
+                }
+#pragma unroll
+            for (int i = 0; i < kStagedChunk; ++i)
+                if (j + i < j_end) {
+                    const float4 p0 = phi_s[(size_t)(j + i) * 32 + lane];
+                    float4 d, p;
+                    p.x = update1(p0.x, dl[i].x, sD.x, mP.x, a, &d.x);
+                    p.y = update1(p0.y, dl[i].y, sD.y, mP.y, a, &d.y);
+                    p.z = update1(p0.z, dl[i].z, sD.z, mP.z, a, &d.z);
+                    p.w = update1(p0.w, dl[i].w, sD.w, mP.w, a, &d.w);
+                    __stcs(reinterpret_cast<float4*>(a.phi + off[i]) + q, p);
+                    __stcs(reinterpret_cast<float4*>(a.delta + off[i]) + q, d);
+                    store_theta4(static_cast<ThetaT*>(a.theta) + off[i], q, p);
+                }
+        }
+    }
+    if ((a.P & 3) && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) scalar_tail<ThetaT>(a, g);
+}
+
 // ---- any subgroup size: two passes over the members -------------------------------------
 //
 // Pass 1 accumulates the two sums; pass 2 re-reads phi_i (the tile was just touched, so this is
@@ -423,6 +579,20 @@ cudaError_t launch_split(const KArgs& k, int groups, int warps, int cluster, int
     return cudaLaunchKernelEx(&cfg, outer_step_split_kernel<MPW, ThetaT, true, MAXW>, k, members_per_cta);
 }
 
+template <typename ThetaT, int WARPS>
+cudaError_t launch_staged(const KArgs& k, int groups, int32_t* status, cudaStream_t stream) {
+    const int64_t quads = (k.P + 3) >> 2;
+    const int64_t tiles = (quads + 31) / 32;
+    if (tiles > 0x7fffffffll) return cudaErrorInvalidConfiguration;
+    const size_t smem = (size_t)k.n * 32 * sizeof(float4);
+    cudaError_t e = cudaFuncSetAttribute(outer_step_staged_kernel<ThetaT, WARPS>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid((unsigned)tiles, (unsigned)groups);
+    outer_step_staged_kernel<ThetaT, WARPS><<<grid, WARPS * 32, smem, stream>>>(k, status);
+    return cudaGetLastError();
+}
+
 template <typename ThetaT>
 cudaError_t launch_any(const KArgs& k, int groups, cudaStream_t stream) {
     const int64_t quads = (k.P + 3) >> 2;
@@ -434,7 +604,7 @@ cudaError_t launch_any(const KArgs& k, int groups, cudaStream_t stream) {
 }
 
 template <typename ThetaT>
-cudaError_t dispatch(const KArgs& k, int groups, cudaStream_t stream) {
+cudaError_t dispatch(const KArgs& k, int groups, int32_t* status, cudaStream_t stream) {
     switch (k.n) {
         case 1:  return launch_reg<1, ThetaT, NOLO_ITEMS_N1>(k, groups, stream);
         // pairs: 2 quads per thread with fp32 theta, 1 with bf16 theta measured best (+0.7 %)
@@ -446,6 +616,10 @@ cudaError_t dispatch(const KArgs& k, int groups, cudaStream_t stream) {
         case 7:  return launch_reg<7, ThetaT, 1>(k, groups, stream);
         case 8:  return launch_reg<8, ThetaT, NOLO_ITEMS_N8>(k, groups, stream);
         default: break;
+    }
+    if (NOLO_STAGED && k.n > kSplitMembersPerCta && k.n <= NOLO_STAGED_MAX_N) {
+        if (k.n <= NOLO_STAGED_SPLIT) return launch_staged<ThetaT, 8>(k, groups, status, stream);
+        return launch_staged<ThetaT, 16>(k, groups, status, stream);
     }
     if (k.n <= kSplitMembersPerCta * kSplitMaxCluster) {
         int cluster = 1;
@@ -480,8 +654,8 @@ cudaError_t launch_outer(const OuterArgs& a, cudaStream_t stream) {
     k.inv_n = 1.0f / (float)a.n;
     const int groups = a.W / a.n;
     if (groups > 65535) return cudaErrorInvalidConfiguration;
-    return a.theta_bf16 ? dispatch<__nv_bfloat16>(k, groups, stream)
-                        : dispatch<float>(k, groups, stream);
+    return a.theta_bf16 ? dispatch<__nv_bfloat16>(k, groups, a.status, stream)
+                        : dispatch<float>(k, groups, a.status, stream);
 }
 
 }  // namespace nolo

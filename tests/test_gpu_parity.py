@@ -34,6 +34,7 @@ def run_both(nolo, W, n, P, seed, step, theta_dtype=torch.float32, stride=None, 
     nolo.nolo_outer_step(h, seed, step)
     torch.cuda.synchronize()
     perm_gpu = nolo.nolo_get_groups(h)
+    assert nolo.nolo_device_status(h) == 0
     nolo.nolo_destroy(h)
 
     perm = O.draw_groups(seed, step, W, n)
@@ -88,12 +89,13 @@ def test_group_sizes_and_ragged_tiles(nolo, n, bf16):
     run_both(nolo, W, n, 5 * 1024 + 3, 7, 3, dt, stride=5 * 1024 + 16)
 
 
-@pytest.mark.parametrize("n", [5, 6, 7, 9, 16, 17, 24, 32, 33, 48, 49, 64, 65, 96, 97, 100, 128, 129, 256, 300, 512, 520])
+@pytest.mark.parametrize("n", [5, 6, 7, 9, 16, 17, 24, 32, 33, 48, 49, 64, 65, 96, 97, 100, 112, 113, 128, 129, 160, 192, 193, 256, 300, 512, 520])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_large_subgroups(nolo, n, bf16):
-    """8 < n <= 512 runs the kernel that splits members across warps and, above 64 members,
-    across a thread-block cluster (with masked member slots when n does not fill them);
-    n > 512 the two-pass kernel.  Two subgroups, ragged P."""
+    """8 < n <= 64 runs the kernel that splits members across warps (with masked member slots
+    when n does not fill them), 64 < n <= 192 the one that stages phi in shared memory with
+    bulk-async copies, up to 512 the thread-block-cluster kernel, above that the two-pass
+    kernel.  Two subgroups, ragged P."""
     dt = torch.bfloat16 if bf16 else torch.float32
     run_both(nolo, 2 * n, n, 1000 + 3, 11, 4, dt)
     if n in (16, 100, 128):
@@ -148,7 +150,7 @@ def test_nan_and_inf_propagate_within_their_subgroup_only(nolo, bf16):
     assert np.array_equal(got_phi[bad & ~np.isnan(want[0])], want[0][bad & ~np.isnan(want[0])])   # signed Inf
 
 
-@pytest.mark.parametrize("W,n", [(4, 2), (8, 8), (24, 12), (72, 72), (130, 130), (600, 600)])
+@pytest.mark.parametrize("W,n", [(4, 2), (8, 8), (24, 12), (72, 72), (130, 130), (200, 200), (600, 600)])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_guard_bands_around_every_buffer_stay_intact(nolo, W, n, bf16):
     """Each state tensor sits between two 4 KiB bands of a known pattern inside a larger
