@@ -331,6 +331,14 @@ int nolo_timing_enable(nolo_handle* h, int enable);
 int nolo_timing_read(nolo_handle* h, int kernel, double* total_ms, int64_t* launches);
 
 /*
+ * Like nolo_timing_read, but returns the distribution of the bracketed
+ * launches since the last read: stats[0..3] = mean, minimum, median and
+ * maximum device time in milliseconds (host array of 4 doubles).  Resets the
+ * record like nolo_timing_read.  Errors: NOLO_EINVAL, NOLO_ENOMEM, NOLO_ECUDA.
+ */
+int nolo_timing_stats(nolo_handle* h, int kernel, double* stats, int64_t* launches);
+
+/*
  * Number of kernels this handle has launched since it was created.
  */
 int nolo_launch_count(nolo_handle* h, int64_t* launches);

@@ -68,6 +68,7 @@ SIGNATURES = {
     "nolo_device_status": [_H, ctypes.POINTER(ctypes.c_int32)],
     "nolo_timing_enable": [_H, _i32],
     "nolo_timing_read": [_H, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)],
+    "nolo_timing_stats": [_H, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)],
     "nolo_launch_count": [_H, ctypes.POINTER(_i64)],
     "nolo_destroy": [_H],
     "nolo_strerror": [_i32],
@@ -278,6 +279,13 @@ def nolo_timing_read(h: Handle, kernel: int):
     ms, cnt = ctypes.c_double(), _i64()
     _check(_lib.nolo_timing_read(h.ptr, kernel, ctypes.byref(ms), ctypes.byref(cnt)), "nolo_timing_read", h)
     return ms.value, cnt.value
+
+
+def nolo_timing_stats(h: Handle, kernel: int):
+    """Returns ({'mean','min','median','max'} in milliseconds, launches) since the last read."""
+    st, cnt = (ctypes.c_double * 4)(), _i64()
+    _check(_lib.nolo_timing_stats(h.ptr, kernel, st, ctypes.byref(cnt)), "nolo_timing_stats", h)
+    return dict(mean=st[0], min=st[1], median=st[2], max=st[3]), cnt.value
 
 
 def nolo_launch_count(h: Handle) -> int:

@@ -458,6 +458,37 @@ int nolo_timing_read(nolo_handle* h, int kernel, double* total_ms, int64_t* laun
     return NOLO_OK;
 }
 
+int nolo_timing_stats(nolo_handle* h, int kernel, double* stats, int64_t* launches) {
+    if (!h) return NOLO_EINVAL;
+    if (kernel < 0 || kernel >= kTimedKernels) return fail(h, NOLO_EINVAL, "unknown kernel id %d", kernel);
+    if (!stats || !launches) return fail(h, NOLO_EINVAL, "output pointers must not be NULL");
+    NOLO_CUDA(h, cudaStreamSynchronize(h->stream));
+    KernelTimer& t = h->timers[kernel];
+    float* ms = new (std::nothrow) float[t.used > 0 ? t.used : 1];
+    if (!ms) return fail(h, NOLO_ENOMEM, "out of host memory");
+    double sum = 0.0;
+    for (int i = 0; i < t.used; ++i) {
+        cudaError_t e = cudaEventElapsedTime(&ms[i], t.start[i], t.stop[i]);
+        if (e != cudaSuccess) { delete[] ms; return cuda_fail(h, e, "cudaEventElapsedTime"); }
+        sum += ms[i];
+    }
+    for (int i = 1; i < t.used; ++i) {            // insertion sort: at most 4096 values
+        const float v = ms[i];
+        int j = i - 1;
+        while (j >= 0 && ms[j] > v) { ms[j + 1] = ms[j]; --j; }
+        ms[j + 1] = v;
+    }
+    const int n = t.used;
+    stats[0] = n ? sum / n : 0.0;
+    stats[1] = n ? ms[0] : 0.0;
+    stats[2] = n ? (n % 2 ? ms[n / 2] : 0.5 * (ms[n / 2 - 1] + ms[n / 2])) : 0.0;
+    stats[3] = n ? ms[n - 1] : 0.0;
+    *launches = n;
+    t.used = 0;
+    delete[] ms;
+    return NOLO_OK;
+}
+
 int nolo_launch_count(nolo_handle* h, int64_t* launches) {
     if (!h || !launches) return NOLO_EINVAL;
     *launches = h->launches;

@@ -460,7 +460,12 @@ def test_timing_and_launch_count(nolo):
     ms, cnt = nolo.nolo_timing_read(h, nolo.NOLO_KERNEL_ROUTE)
     assert cnt == 5 and 0 < ms < 1000
     assert nolo.nolo_timing_read(h, nolo.NOLO_KERNEL_OUTER)[1] == 0
-    assert nolo.nolo_launch_count(h) == 20       # (draw + step) + (draw + copy) per iteration
+    for k in range(4):
+        nolo.nolo_outer_step(h, 0, k)
+    st, cnt = nolo.nolo_timing_stats(h, nolo.NOLO_KERNEL_OUTER)
+    assert cnt == 4 and 0 < st["min"] <= st["median"] <= st["max"] and st["min"] <= st["mean"] <= st["max"]
+    assert nolo.nolo_timing_stats(h, nolo.NOLO_KERNEL_OUTER)[1] == 0
+    assert nolo.nolo_launch_count(h) == 28       # (draw + step) + (draw + copy) per iteration, + 4 more steps
     nolo.nolo_destroy(h)
 
 
