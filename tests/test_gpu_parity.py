@@ -177,6 +177,24 @@ def test_guard_bands_around_every_buffer_stay_intact(nolo, W, n, bf16):
     assert not torch.equal(views[0][:, :P].cpu(), state[0][:, :P])       # and the step did run
 
 
+def test_randomised_shapes(nolo):
+    """Seeded random draw of (W, n, P, stride, dtype, hyper-parameters, seed, step): every kernel
+    path meets odd sizes in combinations the hand-picked cases may miss."""
+    rng = np.random.default_rng(2024)
+    divisors = lambda w: [d for d in range(1, w + 1) if w % d == 0]  # noqa: E731
+    for case in range(48):
+        W = int(rng.choice([1, 2, 3, 4, 6, 8, 10, 12, 16, 18, 30, 36, 64, 70, 90, 96, 130, 144, 200, 260]))
+        n = int(rng.choice(divisors(W)))
+        P = int(rng.choice([1, 3, 6, 31, 127, 129, 640, 1021, 2050, 4097, 9000]))
+        if W * P > 600_000:
+            P = max(1, 600_000 // W)
+        stride = synth.padded_stride(P, 8) + 8 * int(rng.integers(0, 3))
+        dt = torch.bfloat16 if rng.integers(0, 2) else torch.float32
+        hp = tuple(float(np.float32(x)) for x in (rng.uniform(0, 0.95), rng.uniform(0, 1.2), rng.uniform(0, 1.5)))
+        run_both(nolo, W, n, P, int(rng.integers(0, 2**62)), int(rng.integers(0, 2**62)), dt, stride=stride,
+                 hp=hp, state_seed=case)
+
+
 def test_diloco_reduction_on_gpu(nolo):
     """n = W, gamma = 0, shared momentum: all replicas take the same global
     momentum step on the mean outer gradient (Section 3.2)."""
