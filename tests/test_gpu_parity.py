@@ -94,7 +94,7 @@ def test_group_sizes_and_ragged_tiles(nolo, n, bf16):
 def test_large_subgroups(nolo, n, bf16):
     """8 < n <= 64 runs the kernel that splits members across warps (with masked member slots
     when n does not fill them), 64 < n <= 192 the one that stages phi in shared memory with
-    bulk-async copies, up to 512 the thread-block-cluster kernel, above that the two-pass
+    bulk-async copies, up to 256 the thread-block-cluster kernel, above that the two-pass
     kernel.  Two subgroups, ragged P."""
     dt = torch.bfloat16 if bf16 else torch.float32
     run_both(nolo, 2 * n, n, 1000 + 3, 11, 4, dt)
