@@ -5,12 +5,23 @@
 
 One "step" is one pass of the whole path over one batch of synthetic state:
 nolo_outer_step (subgroup draw + fused Eq. 1-3 update) followed by nolo_route
-(route draw + permutation gather of the boundary activations).  The workload is
-the 125M-parameter decoder flattened per worker, W=16 workers in subgroups of
-n=2, float32 phi/delta and bfloat16 theta, with the activations of its
-2-stage / 16-replica layout.  The metric is worker-parameters updated per
-second (W*P per outer step).  With N GPUs, N independent replicas run (the path
-has no cross-GPU exchange); the job's time is the slowest rank's.
+(route draw + permutation gather of the boundary activations).  The headline
+workload is the largest of the paper-shaped configurations that fits the
+device: one pipeline-stage shard of the 6.8B decoder (8 of 32 layers,
+1.61e9 parameters) x W=8 replicas in subgroups of n=2, float32 phi/delta and
+bfloat16 theta (129 GB), with the routing of 32 micro-batches of
+4 x 2048 x 4096 bfloat16 activations across the 3 stage boundaries (12.9 GB).
+If the device has less free memory the 1.3B model (W=8, n=4, all float32,
+126 GB) or the 125M model (W=16, n=2, 20 GB) is taken instead and named in
+`config.workload`.  The metric is worker-parameters updated per second (W*P
+per outer step).  With N GPUs, N independent replicas run (the path has no
+cross-GPU exchange); the job's time is the slowest rank's.  Launched without a
+process launcher, `--gpus N` starts the N rank processes itself.
+
+At N=1 the line also carries `configs`: one record per paper-shaped
+configuration, per kernel path for large subgroups, and for the routing,
+divergence and split-phase kernels, each timed with the library's own CUDA
+event brackets around the kernel.
 
 Prints one JSON line on rank 0.
 """
@@ -18,6 +29,7 @@ Prints one JSON line on rank 0.
 from __future__ import annotations
 
 import argparse
+import concurrent.futures
 import json
 import os
 import subprocess
@@ -35,36 +47,78 @@ from paper_2506_10911_b200 import replicas, synth  # noqa: E402
 
 METRIC = "outer-step params/sec"
 UNIT = "worker-params/s"
-
-# Workload: W=16, n=2, 125M decoder (12 layers, d=768, vocab 50k), bf16 theta.
-W, N_GROUP = 16, 2
-MODEL = "125M"
 ALPHA, BETA, GAMMA = 0.5, 0.7, 0.5
-STAGES = 2                      # the paper's (DP16, PP2) layout of the small model
-MICROBATCH_TOKENS = 4 * 1024    # 4 sequences of 1024 tokens per micro-batch
-BYTES_PER_PARAM = 20            # read phi4+theta2+delta4, write phi4+delta4+theta2
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per worker-parameter of the fused kernel, from the profiler's dram__bytes_read.sum +
-# dram__bytes_write.sum on a 1.34 GB case of the same kernel (W=16, n=2, bf16 theta, P=2^23: 2.6283 GB
-# for 134 217 728 worker-parameters); traffic is proportional to the columns processed.
-PROFILED_DRAM_BYTES_PER_PARAM = 2.6283e9 / (16 * 8388608)
+GB = 1e9
+
+# The paper-shaped workloads, largest first.  tokens = sequences x sequence length per micro-batch.
+WORKLOADS = [
+    dict(name="config 4", W=8, n=2, model="6.8B", stage_of=4, theta="bf16", stages=4, M=32, tokens=4 * 2048,
+         text="one of 4 pipeline-stage shards of the 6.8B decoder (8 layers)"),
+    dict(name="config 3", W=8, n=4, model="1.3B", stage_of=0, theta="f32", stages=1, M=0, tokens=0,
+         text="1.3B decoder flattened"),
+    dict(name="config 2", W=16, n=2, model="125M", stage_of=0, theta="bf16", stages=2, M=16, tokens=4 * 1024,
+         text="125M decoder flattened"),
+]
+
+# DRAM bytes per worker-parameter of the headline kernels from a profiler capture of a small case
+# of the same kernel (dram__bytes_read.sum + dram__bytes_write.sum over the worker-parameters of
+# the captured launch); traffic grows in proportion to the columns processed.  None = not captured
+# since the kernel last changed.
+PROFILED_DRAM_BYTES_PER_PARAM = {
+    "outer_step_reg_kernel<2,bf16,1>": None,
+    "outer_step_reg_kernel<4,float,1>": None,
+}
 
 
-def workload():
-    d = synth.MODEL_SHAPES[MODEL][0]
-    P = synth.model_params(MODEL)
-    return dict(P=P, stride=synth.padded_stride(P), E=MICROBATCH_TOKENS * d, M=W, d=d)
+def bytes_per_param(theta: str) -> int:
+    """Algorithmic bytes per worker-parameter: read phi 4 + theta 4|2 + delta 4, write the same."""
+    return 20 if theta == "bf16" else 24
 
 
-def config_dict(wl, n_gpus):
+def kernel_name(n: int, theta: str) -> str:
+    t = "bf16" if theta == "bf16" else "float"
+    if n <= 8:
+        items = 4 if n == 1 else (2 if (n == 2 and theta != "bf16") else 1)
+        return f"outer_step_reg_kernel<{n},{t},{items}>"
+    if n <= 64:
+        return f"outer_step_split_kernel<{t}> (warps share the subgroup)"
+    if n <= 320:
+        return f"outer_step_twopass_kernel<{t},8 warps,32 quads,4 rows> (second read of phi from L1/L2)"
+    return f"outer_step_twopass_kernel<{t},16 warps,16 quads,8 rows> (second read of phi from L1/L2)"
+
+
+def workload_shape(wl):
+    d = synth.MODEL_SHAPES[wl["model"]][0]
+    P = synth.stage_params(wl["model"], wl["stage_of"]) if wl["stage_of"] else synth.model_params(wl["model"])
+    stride = synth.padded_stride(P)
+    tb = 2 if wl["theta"] == "bf16" else 4
+    E = wl["tokens"] * d
+    act_bytes = (wl["stages"] - 1) * wl["M"] * E * 2           # one copy of the boundary activations, bf16
+    return dict(P=P, stride=stride, d=d, E=E, K=(wl["M"] // wl["W"] if wl["M"] else 0),
+                state_bytes=wl["W"] * stride * (8 + tb), act_bytes=act_bytes)
+
+
+def pick_workload(free_bytes: int, forced: str | None):
+    for wl in WORKLOADS:
+        if forced and wl["name"] != forced:
+            continue
+        sh = workload_shape(wl)
+        need = sh["state_bytes"] + 2 * sh["act_bytes"] + (2 << 30)
+        if forced or need <= free_bytes:
+            return wl, sh
+    raise SystemExit(f"no workload fits {free_bytes / GB:.1f} GB of free device memory")
+
+
+def config_dict(wl, sh, n_gpus):
+    route = (f", outer step + routing of {wl['M']} micro-batches of {wl['tokens']}x{sh['d']} bf16 over "
+             f"{wl['stages']} stages") if wl["M"] else ", outer step (single stage: no routing)"
+    th = "bf16 theta" if wl["theta"] == "bf16" else "fp32 theta"
     return {
-        "workload": f"W={W} n={N_GROUP} {MODEL} decoder flattened (P={wl['P']}), fp32 phi/delta, bf16 theta, "
-                    f"outer step + routing of {wl['M']} micro-batches of {MICROBATCH_TOKENS}x{wl['d']} bf16 "
-                    f"over {STAGES} stages",
-        "W": W, "n": N_GROUP, "P": wl["P"], "stages": STAGES, "microbatches": wl["M"], "E": wl["E"],
-        "alpha": ALPHA, "beta": BETA, "gamma": GAMMA,
-        "replicas": n_gpus,
-        "l2": "state (19.7 GB per replica) is larger than L2; no flush needed",
+        "workload": f"{wl['name']}: W={wl['W']} n={wl['n']} {wl['text']} (P={sh['P']}), fp32 phi/delta, {th}{route}",
+        "W": wl["W"], "n": wl["n"], "P": sh["P"], "stages": wl["stages"], "microbatches": wl["M"], "E": sh["E"],
+        "alpha": ALPHA, "beta": BETA, "gamma": GAMMA, "replicas": n_gpus,
+        "l2": f"state ({sh['state_bytes'] / GB:.1f} GB per replica) is larger than L2; no flush needed",
     }
 
 
@@ -136,69 +190,276 @@ class ClockSampler:
 # reference arm / CPU baseline: the oracle, as it stands, on the host cores
 # ----------------------------------------------------------------------------
 
-def oracle_sample_state(cols: int, seed: int = 0):
+def host_cores() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except Exception:
+        return max(1, os.cpu_count() or 1)
+
+
+def oracle_sample_state(wl, sh, cols: int, seed: int = 0):
     """The first `cols` columns of the workload's state and the matching share of its routed
     activations, as numpy arrays (bfloat16 as uint16 bit patterns)."""
-    wl = workload()
-    phi, theta, delta = synth.make_state(W, cols, seed, torch.bfloat16)
-    e_s = max(1, int(wl["E"] * cols / wl["P"]))
-    acts = synth.make_acts(STAGES - 1, W, wl["M"] // W, e_s, 1000 + seed, torch.bfloat16)
+    tdt = torch.bfloat16 if wl["theta"] == "bf16" else torch.float32
+    phi, theta, delta = synth.make_state(wl["W"], cols, seed, tdt)
     as_np = lambda x: x.view(torch.int16).numpy().view(np.uint16) if x.dtype == torch.bfloat16 else x.numpy()  # noqa: E731
-    return [as_np(x) for x in (phi, theta, delta, acts)]
+    out = [as_np(x) for x in (phi, theta, delta)]
+    if wl["M"]:
+        e_s = max(1, int(sh["E"] * cols / sh["P"]))
+        acts = synth.make_acts(wl["stages"] - 1, wl["W"], sh["K"], e_s, 1000 + seed, torch.bfloat16)
+        out.append(as_np(acts))
+    else:
+        out.append(None)
+    return out
 
 
-def time_oracle_step(state, k: int) -> float:
-    """One step of the oracle as it stands: outer step, then routing."""
+def oracle_step(wl, state, k: int, threads: int = 1) -> float:
+    """One step of the oracle as it stands: outer step, then routing.  With threads > 1 the
+    columns are cut into chunks and the same oracle function runs on each chunk in a thread pool
+    (the step is independent per column; numpy releases the interpreter lock in its loops)."""
     from oracle import nolo_oracle as O
+    W, n = wl["W"], wl["n"]
+    dt = O.THETA_BF16 if wl["theta"] == "bf16" else O.THETA_F32
     t0 = time.perf_counter()
-    O.outer_step_seeded(state[0], state[1], state[2], k, k, N_GROUP, ALPHA, BETA, GAMMA, O.THETA_BF16)
-    O.route_forward(state[3], O.draw_route(k, k, STAGES, W, state[3].shape[2]))
+    perm = O.draw_groups(k, k, W, n)
+    phi, theta, delta, acts = state
+    table = O.draw_route(k, k, wl["stages"], W, sh_k(acts)) if acts is not None else None
+    if threads <= 1:
+        O.outer_step(phi, theta, delta, perm, n, ALPHA, BETA, GAMMA, dt)
+        if acts is not None:
+            O.route_forward(acts, table)
+    else:
+        cols = phi.shape[1]
+        edges = np.linspace(0, cols, 4 * threads + 1).astype(np.int64)
+        jobs = [(int(a), int(b)) for a, b in zip(edges[:-1], edges[1:]) if b > a]
+        with concurrent.futures.ThreadPoolExecutor(threads) as pool:
+            fut = [pool.submit(O.outer_step, phi[:, a:b], theta[:, a:b], delta[:, a:b], perm, n, ALPHA, BETA, GAMMA, dt)
+                   for a, b in jobs]
+            if acts is not None:
+                e = acts.shape[3]
+                ee = np.linspace(0, e, threads + 1).astype(np.int64)
+                fut += [pool.submit(O.route_forward, acts[..., int(a):int(b)], table)
+                        for a, b in zip(ee[:-1], ee[1:]) if b > a]
+            for f in fut:
+                f.result()
     return time.perf_counter() - t0
 
 
-def cpu_baseline(cols: int = 1 << 24):
-    """One oracle step on the first `cols` columns x all W rows."""
-    state = oracle_sample_state(cols)
-    dt = time_oracle_step(state, 0)
-    return {"value": W * cols / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"1 step (outer step + routing) on {cols} of {workload()['P']} columns x {W} workers "
-                      f"(numpy float64, single thread), {dt:.1f} s"}
+def sh_k(acts) -> int:
+    return acts.shape[2]
+
+
+def cpu_baseline(wl, sh, cols: int):
+    """One oracle step on the first `cols` columns x all W rows: once on one thread, once with
+    the columns spread over all host cores."""
+    state = oracle_sample_state(wl, sh, cols)
+    cores = host_cores()
+    t1 = oracle_step(wl, state, 0, 1)
+    tc = oracle_step(wl, state, 0, cores) if cores > 1 else t1
+    W = wl["W"]
+    what = "outer step + routing" if wl["M"] else "outer step"
+    return {"value": W * cols / tc, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"1 step ({what}) on {cols} of {sh['P']} columns x {W} workers, numpy float64: "
+                      f"{tc:.1f} s with the columns spread over {cores} threads, {t1:.1f} s on one thread",
+            "single_thread": {"value": W * cols / t1, "unit": UNIT, "cores": 1}}
 
 
 def run_reference(args):
     rank, _, world = replicas.env_rank()
     if rank != 0:
-        return
-    wl = workload()
-    probe = oracle_sample_state(1 << 14)
-    t_probe = min(time_oracle_step(probe, 0) for _ in range(2)) / (1 << 14)   # seconds per column
+        return 0
+    wl = next(w for w in WORKLOADS if w["name"] == (args.workload or WORKLOADS[0]["name"]))
+    sh = workload_shape(wl)
+    cores = host_cores()
+    probe = oracle_sample_state(wl, sh, 1 << 16)
+    t_probe = min(oracle_step(wl, probe, 0, cores) for _ in range(2)) / (1 << 16)   # seconds per column
     budget = 120.0 / max(1, args.steps + args.warmup)
-    cols = int(min(1 << 22, max(1 << 12, budget / t_probe)))
-    state = oracle_sample_state(cols)
+    cols = int(min(1 << 24, max(1 << 12, budget / t_probe)))
+    state = oracle_sample_state(wl, sh, cols)
     for k in range(args.warmup):
-        time_oracle_step(state, k)
+        oracle_step(wl, state, k, cores)
     t0 = time.perf_counter()
     for k in range(args.steps):
-        time_oracle_step(state, k)
+        oracle_step(wl, state, k, cores)
     dt = time.perf_counter() - t0
+    W = wl["W"]
     value = W * cols * args.steps / dt
-    sample = (f"each step = 1 oracle step (outer step + routing) on {cols} of {wl['P']} columns x {W} workers "
-              f"(numpy float64, 1 thread)")
+    what = "outer step + routing" if wl["M"] else "outer step"
+    sample = (f"each step = 1 oracle step ({what}) on {cols} of {sh['P']} columns x {W} workers "
+              f"(numpy float64, columns spread over {cores} threads)")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": config_dict(wl, world),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "config": config_dict(wl, sh, world),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+    return 0
 
 
 # ----------------------------------------------------------------------------
 # our arm
 # ----------------------------------------------------------------------------
+
+def alloc_state(W, stride, theta, dev):
+    tdt = torch.bfloat16 if theta == "bf16" else torch.float32
+    return (torch.empty((W, stride), dtype=torch.float32, device=dev),
+            torch.empty((W, stride), dtype=tdt, device=dev),
+            torch.empty((W, stride), dtype=torch.float32, device=dev))
+
+
+def stats_record(name, kernel, stats, cnt, nbytes, peak, copy_gbs, **extra):
+    gbs = nbytes / (stats["mean"] * 1e-3) / GB if cnt and stats["mean"] > 0 else None
+    rec = {"name": name, "kernel": kernel, **extra, "launches_timed": cnt,
+           "ms_per_launch": stats["mean"], "ms_per_launch_min": stats["min"], "ms_per_launch_max": stats["max"],
+           "bytes_per_launch": nbytes, "gbs": gbs, "frac": gbs / peak if gbs else None,
+           "frac_of_same_run_copy": gbs / copy_gbs if gbs and copy_gbs else None}
+    return rec
+
+
+def time_outer_cases(nolo, dev, W, P, theta, variants, peak, copy_gbs, warmup=3, drift="normal",
+                     extra_records=False):
+    """Allocate and fill one state, then time the outer step for each (name, n, gamma, steps) in
+    `variants` on it; returns the records."""
+    stride = synth.padded_stride(P)
+    need = W * stride * (8 + (2 if theta == "bf16" else 4))
+    free = torch.cuda.mem_get_info()[0]
+    if need > 0.97 * free:
+        return [{"name": v[0], "skipped": f"needs {need / GB:.1f} GB, {free / GB:.1f} GB free"} for v in variants]
+    phi, th, delta = alloc_state(W, stride, theta, dev)
+    synth.fill_state_(phi, th, delta, P, seed=1, drift=drift)
+    recs = []
+    for name, n, gamma, steps in variants:
+        h = nolo.nolo_create(W, n, P, 1, ALPHA, BETA, gamma)
+        nolo.nolo_bind_state(h, phi, th, delta)
+        for k in range(warmup):
+            nolo.nolo_outer_step(h, k, k)
+        torch.cuda.synchronize()
+        nolo.nolo_timing_enable(h, True)
+        for k in range(steps):
+            nolo.nolo_outer_step(h, warmup + k, warmup + k)
+        st, cnt = nolo.nolo_timing_stats(h, nolo.NOLO_KERNEL_OUTER)
+        recs.append(stats_record(name, kernel_name(n, theta), st, cnt, bytes_per_param(theta) * W * P, peak,
+                                 copy_gbs, W=W, n=n, P=P, theta=theta, resident_gb=need / GB,
+                                 params_per_s=W * P / (st["mean"] * 1e-3)))
+        if extra_records:
+            # replica-divergence metric on the same state (read-only, 4 B per worker-parameter)
+            for _ in range(steps):
+                nolo.nolo_divergence(h)
+            st, cnt = nolo.nolo_timing_stats(h, nolo.NOLO_KERNEL_DIVERGENCE)
+            recs.append(stats_record(f"{name}: divergence", "divergence_partial_kernel + divergence_final_kernel",
+                                     st, cnt, 4 * W * P, peak, copy_gbs, W=W, P=P,
+                                     note="read-only pass; the read-only ceiling is above the copy figure"))
+            # split-phase step: subgroup means of phi prepared ahead, then the step that uses them
+            mean = torch.empty((W // n, stride), dtype=torch.float64, device=dev)
+            nolo.nolo_bind_prepared(h, mean)
+            for k in range(steps):
+                nolo.nolo_outer_prepare(h, 77, k)
+                nolo.nolo_outer_step_prepared(h, 77, k)
+            sp, cp = nolo.nolo_timing_stats(h, nolo.NOLO_KERNEL_PREPARE)
+            so, co = nolo.nolo_timing_stats(h, nolo.NOLO_KERNEL_OUTER)
+            recs.append(stats_record(f"{name}: split-phase prepare", "group_mean_kernel", sp, cp,
+                                     int((4 + 8 / n) * W * P), peak, copy_gbs, W=W, n=n, P=P,
+                                     note="reads phi (4 B), writes float64 subgroup means (8/n B) per "
+                                          "worker-parameter"))
+            recs.append(stats_record(f"{name}: split-phase step", kernel_name(n, theta) + " with prepared means",
+                                     so, co, int((bytes_per_param(theta) + 8 / n) * W * P), peak, copy_gbs,
+                                     W=W, n=n, P=P,
+                                     note="the fused step's bytes plus the float64 means (8/n B per "
+                                          "worker-parameter)"))
+            del mean
+        nolo.nolo_destroy(h)
+    del phi, th, delta
+    torch.cuda.empty_cache()
+    return recs
+
+
+def extra_configs(nolo, dev, peak, copy_gbs, args):
+    """One record per paper-shaped configuration other than the headline, per large-subgroup
+    kernel path, and for the NEXT kernels.  N=1 only."""
+    out = []
+    run = lambda *a, **kw: out.extend(time_outer_cases(nolo, dev, *a, peak=peak, copy_gbs=copy_gbs, **kw))  # noqa: E731
+    run(4, 1 << 20, "f32", [("config 1: W=4 n=2 P=2^20 fp32 (state 50 MB: partly L2-resident)", 2, GAMMA, 20)])
+    run(16, synth.model_params("125M"), "bf16", [("config 2: W=16 n=2 125M decoder, bf16 theta", 2, GAMMA, 10)],
+        extra_records=True)
+    run(8, synth.model_params("1.3B"), "f32",
+        [(f"config 3: W=8 n=4 1.3B decoder fp32, gamma={g}", 4, g, 3) for g in (0.0, 0.5)])
+    if "config 4" not in args.headline:
+        run(8, synth.stage_params("6.8B", 4), "bf16", [("config 4: W=8 n=2 6.8B/4 stage shard, bf16 theta", 2, GAMMA, 3)])
+    for W in (8, 32, 128):
+        run(W, 1 << 26, "f32", [(f"config 5: W={W} n={n} P=2^26 fp32, Student-t(3) drift", n, GAMMA, 3)
+                                for n in (2, 4, 8)], drift="student_t3")
+    for n in (16, 32, 64, 96, 128, 192, 256, 512, 1024):
+        for theta in ("f32", "bf16"):
+            P = max(1 << 16, ((3 << 28) // n) & ~63)           # about 3.2e9 bytes of phi
+            run(n, P, theta, [(f"large_n: one subgroup of n=W={n}, P={P}, {theta} theta (DiLoCo mode)", n, GAMMA, 5)])
+    return out
+
+
+def measure_e2e(nolo, args, wl, sh, state, acts, acts_out, world, dev):
+    """End to end: state and activations in pinned host memory, through the host entry points.
+    The full state (>100 GB) cannot be page-locked on the host, so a column slice of it is
+    streamed: the first e2e_cols columns of every worker and the same share of every activation.
+    Returns (record, note)."""
+    phi, theta, delta = state
+    W, n, P, E, M, K = wl["W"], wl["n"], sh["P"], sh["E"], wl["M"], sh["K"]
+    try:
+        import psutil
+        host_free = psutil.virtual_memory().available
+    except Exception:
+        host_free = 32 << 30
+    tb = 2 if wl["theta"] == "bf16" else 4
+    cols = min(P, args.e2e_cols)
+    while cols > (1 << 20) and world * W * cols * (8 + tb) * 1.3 > 0.4 * host_free:
+        cols //= 2
+    cols &= ~63
+    e_s = max(64, (int(E * cols / P) & ~63)) if M else 0
+    try:
+        hh = nolo.nolo_create(W, n, cols, wl["stages"], ALPHA, BETA, GAMMA)
+        nolo.nolo_bind_state(hh, phi, theta, delta)            # same rows, first `cols` columns
+        h_state = [torch.empty((W, cols), dtype=x.dtype, pin_memory=True) for x in state]
+        for hs, ds in zip(h_state, state):
+            hs.copy_(ds[:, :cols])
+        if M:
+            shape = (wl["stages"] - 1, W, K, e_s)
+            d_in = acts.view(-1)[:int(np.prod(shape))].view(shape)
+            d_out = acts_out.view(-1)[:int(np.prod(shape))].view(shape)
+            h_acts = torch.empty(shape, dtype=acts.dtype, pin_memory=True).copy_(d_in)
+            h_out = torch.empty(shape, dtype=acts.dtype, pin_memory=True)
+            nolo.nolo_bind_route(hh, M, e_s, d_out)
+
+        def e2e_step(k):
+            nolo.nolo_outer_step_host(hh, k, k, *h_state, host_stride=cols)
+            if M:
+                nolo.nolo_route_host(hh, k, k, h_acts, h_out, d_in)
+
+        e2e_step(0)
+        replicas.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for k in range(args.e2e_steps):
+            e2e_step(1 + k)
+        torch.cuda.synchronize()
+        e2e_ms = (time.perf_counter() - t0) * 1e3
+        replicas.barrier()
+        j_ms, j_units = replicas.job_time_and_units(e2e_ms, float(W) * cols * args.e2e_steps, dev)
+        state_bytes = W * cols * (8 + tb)
+        act_bytes = (h_acts.numel() * h_acts.element_size()) if M else 0
+        rec = {"value": replicas.throughput(j_units, j_ms), "unit": UNIT,
+               "h2d_bytes_per_step": state_bytes + act_bytes, "d2h_bytes_per_step": state_bytes + act_bytes,
+               "steps": args.e2e_steps, "ms_per_step": j_ms / args.e2e_steps,
+               "slice": f"the first {cols} of {P} columns of all {W} workers and the same share of every "
+                        f"activation ({e_s} of {E} elements): the whole state cannot be page-locked on the host",
+               "api": "nolo_outer_step_host + nolo_route_host (pinned host buffers, chunked copies "
+                      "overlapped with the kernel)"}
+        nolo.nolo_destroy(hh)
+        return rec, None
+    except Exception as ex:   # e.g. not enough page-lockable host memory
+        return None, f"{type(ex).__name__}: {ex}"
+
 
 def run_ours(args):
     from paper_2506_10911_b200 import build
@@ -211,24 +472,38 @@ def run_ours(args):
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     replicas.init("nccl", dev)
+    peak, peak_kind = measured_peak()
 
-    wl = workload()
-    P, stride, E, M = wl["P"], wl["stride"], wl["E"], wl["M"]
-    K = M // W
-    phi = torch.empty((W, stride), dtype=torch.float32, device=dev)
-    theta = torch.empty((W, stride), dtype=torch.bfloat16, device=dev)
-    delta = torch.empty((W, stride), dtype=torch.float32, device=dev)
+    # ---- a plain copy of our own in the same run, as context for the roofline fraction
+    copy_gbs = None
+    try:
+        nbytes = 4 << 30
+        src = torch.empty(nbytes, dtype=torch.uint8, device=dev).fill_(1)
+        dst = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        copy_gbs = nolo.nolo_copy_probe(src, dst, nbytes, 10)
+        del src, dst
+        torch.cuda.empty_cache()
+    except Exception:
+        copy_gbs = None
+
+    wl, sh = pick_workload(torch.cuda.mem_get_info()[0], args.workload)
+    W, n, P, stride, E, M, K = wl["W"], wl["n"], sh["P"], sh["stride"], sh["E"], wl["M"], sh["K"]
+    phi, theta, delta = alloc_state(W, stride, wl["theta"], dev)
     synth.fill_state_(phi, theta, delta, P, seed=rank)
-    acts = synth.make_acts(STAGES - 1, W, K, E, seed=1000 + rank, dtype=torch.bfloat16, device=dev)
-    acts_out = torch.empty_like(acts)
+    acts = acts_out = None
+    if M:
+        acts = synth.make_acts(wl["stages"] - 1, W, K, E, seed=1000 + rank, dtype=torch.bfloat16, device=dev)
+        acts_out = torch.empty_like(acts)
 
-    h = nolo.nolo_create(W, N_GROUP, P, STAGES, ALPHA, BETA, GAMMA)
+    h = nolo.nolo_create(W, n, P, wl["stages"], ALPHA, BETA, GAMMA)
     nolo.nolo_bind_state(h, phi, theta, delta)
-    nolo.nolo_bind_route(h, M, E, acts_out)
+    if M:
+        nolo.nolo_bind_route(h, M, E, acts_out)
 
     def step(k):
         nolo.nolo_outer_step(h, k, k)
-        nolo.nolo_route(h, k, k, acts)
+        if M:
+            nolo.nolo_route(h, k, k, acts)
 
     for k in range(args.warmup):
         step(k)
@@ -252,124 +527,98 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     local_ms = e0.elapsed_time(e1)
     outer_stats, outer_cnt = nolo.nolo_timing_stats(h, nolo.NOLO_KERNEL_OUTER)
-    outer_ms = outer_stats["mean"] * outer_cnt
-    route_ms, route_cnt = nolo.nolo_timing_read(h, nolo.NOLO_KERNEL_ROUTE)
-    nolo.nolo_timing_enable(h, False)
+    route_stats, route_cnt = nolo.nolo_timing_stats(h, nolo.NOLO_KERNEL_ROUTE)
     launches = nolo.nolo_launch_count(h) - launches0
     job_ms, job_units = replicas.job_time_and_units(local_ms, float(W) * P * args.steps, dev)
     value = replicas.throughput(job_units, job_ms)
 
-    # ---- a plain copy of our own in the same run, as context for the roofline fraction
-    copy_gbs = None
-    if rank == 0:
-        try:
-            nbytes = 4 << 30
-            src = torch.empty(nbytes, dtype=torch.uint8, device=dev).fill_(1)
-            dst = torch.empty(nbytes, dtype=torch.uint8, device=dev)
-            copy_gbs = nolo.nolo_copy_probe(src, dst, nbytes, 10)
-            del src, dst
-        except Exception:
-            copy_gbs = None
+    # ---- backward routing of the same activations (gradients return along the same path)
+    back_stats = back_cnt = None
+    if M and rank == 0 and world == 1:
+        for k in range(5):
+            nolo.nolo_route_backward(h, k, k, acts_out, acts)
+        back_stats, back_cnt = nolo.nolo_timing_stats(h, nolo.NOLO_KERNEL_ROUTE)
+    nolo.nolo_timing_enable(h, False)
 
-    # ---- end to end: state and activations in pinned host memory, through the host entry points
-    e2e = None
-    e2e_note = None
-    host_need = world * (W * stride * 10 + 2 * acts.numel() * acts.element_size())
-    try:
-        import psutil
-        host_free = psutil.virtual_memory().available
-    except Exception:
-        host_free = None
-    if not args.no_e2e and host_free is not None and host_need > 0.5 * host_free:
-        e2e_note = (f"skipped: page-locking {host_need / 1e9:.0f} GB for {world} replicas would take more than "
-                    f"half of the {host_free / 1e9:.0f} GB of free host memory")
-    elif not args.no_e2e:
-        try:
-            h_state = [torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for x in (phi, theta, delta)]
-            for hs, ds in zip(h_state, (phi, theta, delta)):
-                hs.copy_(ds)
-            h_acts = torch.empty(acts.shape, dtype=acts.dtype, pin_memory=True).copy_(acts)
-            h_out = torch.empty(acts.shape, dtype=acts.dtype, pin_memory=True)
-
-            def e2e_step(k):
-                nolo.nolo_outer_step_host(h, k, k, *h_state, host_stride=stride)
-                nolo.nolo_route_host(h, k, k, h_acts, h_out, acts)
-
-            e2e_step(0)
-            replicas.barrier()
-            torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            for k in range(args.e2e_steps):
-                e2e_step(1 + k)
-            torch.cuda.synchronize()
-            e2e_ms = (time.perf_counter() - t0) * 1e3
-            replicas.barrier()
-            j_ms, j_units = replicas.job_time_and_units(e2e_ms, float(W) * P * args.e2e_steps, dev)
-            state_bytes = W * P * (4 + 2 + 4)
-            act_bytes = acts.numel() * acts.element_size()
-            e2e = {"value": replicas.throughput(j_units, j_ms), "unit": UNIT,
-                   "h2d_bytes_per_step": state_bytes + act_bytes, "d2h_bytes_per_step": state_bytes + act_bytes,
-                   "steps": args.e2e_steps, "ms_per_step": j_ms / args.e2e_steps,
-                   "api": "nolo_outer_step_host + nolo_route_host (pinned host buffers, chunked copies "
-                          "overlapped with the kernel)"}
-            del h_state, h_acts, h_out
-        except Exception as ex:   # e.g. not enough page-lockable host memory
-            e2e_note = f"{type(ex).__name__}: {ex}"
+    e2e, e2e_note = (None, "skipped") if args.no_e2e else measure_e2e(
+        nolo, args, wl, sh, (phi, theta, delta), acts, acts_out, world, dev)
 
     if rank != 0:
         nolo.nolo_destroy(h)
-        return
+        return 0
 
-    peak, peak_kind = measured_peak()
-    per_launch_ms = outer_ms / max(1, outer_cnt)
-    achieved = BYTES_PER_PARAM * W * P / (per_launch_ms * 1e-3) / 1e9
-    route_bytes = 2 * acts.numel() * acts.element_size()
+    kname = kernel_name(n, wl["theta"])
+    bpp = bytes_per_param(wl["theta"])
+    per_launch_ms = outer_stats["mean"]
+    achieved = bpp * W * P / (per_launch_ms * 1e-3) / GB
+    dram_bpp = PROFILED_DRAM_BYTES_PER_PARAM.get(kname)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": job_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": config_dict(wl, world),
+        "config": config_dict(wl, sh, world),
         "hbm_gbs": achieved, "pct_of_8tbs_nominal": achieved / 8000.0,
         "clocks": clocks,
         "e2e": e2e if e2e is not None else {"value": None, "unit": UNIT, "note": e2e_note or "skipped"},
         "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "kernel": "outer_step_reg_kernel<2,bf16,1>", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": kname, "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "traffic": PROFILED_DRAM_BYTES_PER_PARAM * W * P,
-                     "traffic_note": "ncu dram bytes of a 1.34 GB case of this kernel scaled by columns",
-                     "bytes_per_launch": BYTES_PER_PARAM * W * P,
+                     "frac_of_same_run_copy": achieved / copy_gbs if copy_gbs else None,
+                     "frac_note": "peak is a plain torch copy measured earlier on this pool; our own one-shot "
+                                  "128-bit copy timed in this run is the tighter ceiling (frac_of_same_run_copy)",
+                     "traffic": dram_bpp * W * P if dram_bpp else None,
+                     "traffic_note": "profiler dram bytes of a small case of this kernel scaled by columns"
+                                     if dram_bpp else "not captured since the kernel last changed",
+                     "bytes_per_launch": bpp * W * P,
                      "ms_per_launch": per_launch_ms, "ms_per_launch_min": outer_stats["min"],
                      "ms_per_launch_median": outer_stats["median"], "ms_per_launch_max": outer_stats["max"],
                      "launches_timed": outer_cnt,
                      "plain_copy_same_run_gbs": copy_gbs},
-        "route": {"ms_per_launch": route_ms / max(1, route_cnt), "bytes_per_launch": route_bytes,
-                  "achieved_gbs": route_bytes / (route_ms / max(1, route_cnt) * 1e-3) / 1e9 if route_ms else None},
     }
+    if M:
+        rb = 2 * acts.numel() * acts.element_size()
+        line["route"] = stats_record("routing, forward, all boundaries", "route_copy16_kernel", route_stats, route_cnt,
+                                     rb, peak, copy_gbs)
+        if back_stats is not None:
+            line["route_backward"] = stats_record("routing, backward, all boundaries", "route_copy16_kernel",
+                                                  back_stats, back_cnt, rb, peak, copy_gbs)
+    nolo.nolo_destroy(h)
+    del phi, theta, delta, acts, acts_out
+    torch.cuda.empty_cache()
+    if world == 1 and not args.no_configs:
+        args.headline = wl["name"]
+        line["configs"] = extra_configs(nolo, dev, peak, copy_gbs, args)
     if args.no_cpu_baseline or world > 1:
         line["cpu_baseline"] = None
     else:
-        line["cpu_baseline"] = cpu_baseline(args.cpu_cols)
-    nolo.nolo_destroy(h)
+        line["cpu_baseline"] = cpu_baseline(wl, sh, args.cpu_cols)
     print(json.dumps(line), flush=True)
+    return 0
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=[w["name"] for w in WORKLOADS], default=None,
+                    help="force a workload instead of taking the largest that fits")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-cols", type=int, default=1 << 26)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration records")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-cols", type=int, default=1 << 24)
+    ap.add_argument("--cpu-cols", type=int, default=1 << 25)
     args = ap.parse_args()
     args.warmup = max(3, args.warmup)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not under a launcher: start the N rank processes ourselves (one per GPU)
+        return replicas.launch(args.gpus, [sys.executable, os.path.abspath(__file__), *sys.argv[1:]])
     if args.impl == "reference":
-        run_reference(args)
-    else:
-        run_ours(args)
+        return run_reference(args)
+    return run_ours(args)
 
 
 if __name__ == "__main__":
-    main()
+    raise SystemExit(main())

@@ -52,6 +52,9 @@ extern "C" {
 #define NOLO_KERNEL_OUTER 0 /* kernel ids for nolo_timing_read() */
 #define NOLO_KERNEL_ROUTE 1
 #define NOLO_KERNEL_DIVERGENCE 2
+#define NOLO_KERNEL_PREPARE 3
+
+#define NOLO_SIM_MAX_SAMPLES (1LL << 40)  /* W*H*T*trials limit of nolo_sim_straggler */
 
 typedef struct nolo_handle nolo_handle;
 
@@ -98,11 +101,46 @@ int nolo_bind_state(nolo_handle* h, void* phi, void* theta, void* delta,
  *   4. delta_i <- alpha delta_i - beta mean_G(Delta) - gamma (phi_i - mean_G(phi))   (Eq. 2)
  *      phi_i   <- phi_i + delta_i                                                    (Eq. 3)
  *      theta_i <- phi_i  (rounded to nearest-even when theta is bfloat16).
- * float32 arithmetic; every element of every worker is read once and written
- * once.  Asynchronous.  Errors: NOLO_EINVAL (NULL handle), NOLO_ESTATE (no
+ * float32 arithmetic, with the subgroup mean of phi carried to about 46 bits so
+ * that gamma (phi_i - mean) is accurate for weights of any magnitude; sums in a
+ * fixed order (results are reproducible bit for bit); every element of every
+ * worker is fetched from device memory once and written once.  Asynchronous.  Errors: NOLO_EINVAL (NULL handle), NOLO_ESTATE (no
  * state bound), NOLO_ECUDA (launch failure).
  */
 int nolo_outer_step(nolo_handle* h, uint64_t seed, uint64_t step);
+
+/*
+ * The outer step in two phases (Section 3.2, the remark after Eq. 3: the slow
+ * weights of the partners are known once the previous outer step is done, so
+ * they can be communicated then, overlapped with the inner phase; only the
+ * pseudo-gradients have to be exchanged at the step itself).
+ *
+ * nolo_bind_prepared attaches the buffer that carries the early part:
+ *   mean_phi     device, float64 [W/n][mean_stride], 16-byte aligned, borrowed,
+ *                disjoint from the state; row g receives the mean of phi over
+ *                subgroup g.  float64 so that gamma (phi_i - mean) loses
+ *                nothing to the rounding of the mean.
+ *   mean_stride  elements between rows; >= P and a multiple of 8.
+ * nolo_outer_prepare(seed, next_step) draws the partition that step
+ * `next_step` will use (the draw is a pure function of (seed, step), so it is
+ * known in advance) and writes mean_phi[g][p] = (1/n) sum_{j in G_g} phi_j[p]
+ * from the current phi.  Read-only on the state.  Call it after the last
+ * change of phi, e.g. right after the previous outer step, on the same stream.
+ * nolo_outer_step_prepared(seed, step) is nolo_outer_step with the mean of phi
+ * in Eq. 2 taken from mean_phi instead of being reduced again; it still forms
+ * Delta_j = phi_j - theta_j and its subgroup sum.  It returns NOLO_ESTATE and
+ * does nothing when no means are prepared, when they were prepared for another
+ * (seed, step), or when an outer step of this handle has changed phi since
+ * (phi changed by the caller behind the library's back cannot be detected).
+ * Results equal nolo_outer_step's to float32 rounding.  On one GPU this form
+ * moves more bytes than the fused step (it reads phi once more and the means);
+ * it is the building block for a worker-sharded deployment, where the early
+ * exchange hides behind the inner phase.
+ * Asynchronous.  Errors: NOLO_EINVAL, NOLO_EALIGN, NOLO_ESTATE, NOLO_ECUDA.
+ */
+int nolo_bind_prepared(nolo_handle* h, void* mean_phi, int64_t mean_stride);
+int nolo_outer_prepare(nolo_handle* h, uint64_t seed, uint64_t next_step);
+int nolo_outer_step_prepared(nolo_handle* h, uint64_t seed, uint64_t step);
 
 /*
  * (No counterpart in the paper: this is a packaging variant of nolo_outer_step.)
@@ -288,7 +326,10 @@ double nolo_expected_pair_exchange(double mu, double sigma);
  *   host_stats   host, 4 doubles: mean time with the global barrier, mean time
  *           with subgroup waits, then the standard errors of the two means
  *   host_trials  host, [trials][2] (barrier, subgroup) per trial, or NULL
- * Synchronous; allocates and frees its own scratch.  trials 1..2^20.
+ * Synchronous; allocates and frees its own scratch.  trials 1..2^20, and the
+ * total number of samples W*H*T*trials at most NOLO_SIM_MAX_SAMPLES (2^40, about
+ * 20 s of GPU time): a larger request is refused with NOLO_EINVAL rather than
+ * left to occupy the device.
  * Errors: NOLO_EINVAL, NOLO_ENOMEM, NOLO_ECUDA.
  */
 int nolo_sim_straggler(int W, int n, int H, int T, double mu, double sigma, int64_t trials,
@@ -309,23 +350,13 @@ int nolo_copy_probe(const void* src, void* dst, int64_t bytes, int iters, void* 
                     double* ms_per_copy);
 
 /*
- * Device-side status of this handle's kernels.  The outer-step kernel for
- * subgroups of 65 to 192 members waits on a shared-memory barrier for its
- * bulk copies; that wait is bounded, and a CTA whose wait ever ran out leaves
- * its tile of the state untouched and raises this word instead of hanging.
- *   host_out  receives 0 (nothing happened) or 1 (a wait ran out since the
- *             handle was created: the last outer steps are incomplete)
- * Synchronises the stream.  Errors: NOLO_EINVAL, NOLO_ECUDA.
- */
-int nolo_device_status(nolo_handle* h, int32_t* host_out);
-
-/*
  * Device-time instrumentation.  With enable != 0 every later launch of the
- * fused outer-step kernel, the routing copy kernel and the divergence kernels is bracketed by CUDA
+ * fused outer-step kernel, the routing copy kernel, the divergence kernels and the
+ * subgroup-mean kernel of nolo_outer_prepare is bracketed by CUDA
  * events on the bound stream (up to 4096 launches per kernel between reads).
  * nolo_timing_read synchronises the stream, returns the summed device time in
  * milliseconds and the number of bracketed launches of `kernel`
- * (NOLO_KERNEL_OUTER / NOLO_KERNEL_ROUTE / NOLO_KERNEL_DIVERGENCE) since the last read, and resets them.
+ * (NOLO_KERNEL_OUTER / _ROUTE / _DIVERGENCE / _PREPARE) since the last read, and resets them.
  */
 int nolo_timing_enable(nolo_handle* h, int enable);
 int nolo_timing_read(nolo_handle* h, int kernel, double* total_ms, int64_t* launches);

@@ -12,6 +12,9 @@ values, closed forms and invariants):
                          momentum over a subgroup of n workers) and Eq. 3
                          (slow-weight update), then the reset of the fast
                          weights to the new slow weights (Section 3.2).
+* ``subgroup_mean_phi`` -- the subgroup mean of the slow weights inside Eq. 2,
+                         on its own (the part Section 3.2 says can be
+                         exchanged ahead of the step).
 * ``divergence``      -- the replica spread plotted in Fig. 3b (standard
                          deviation of the weights across the data-parallel
                          replicas).
@@ -198,6 +201,23 @@ def outer_step(phi, theta, delta, perm, n, alpha, beta, gamma, theta_dtype=THETA
     else:
         theta_new = phi_new.copy()
     return phi_new, delta_new, theta_new
+
+
+def subgroup_mean_phi(phi, perm, n):
+    """The part of Eq. 2 that depends on the slow weights alone: for every
+    subgroup g, mean_g[p] = (1/n) * sum_{j in G_g} phi_j[p], float64 [W/n, P].
+
+    Section 3.2 (the remark after Eq. 3) points out that these slow weights
+    are known when the previous outer step ends and can be exchanged then.
+    """
+    phi = np.asarray(phi)
+    W, P = phi.shape
+    perm = np.asarray(perm)
+    out = np.empty((W // n, P), dtype=np.float64)
+    for g in range(W // n):
+        members = [int(w) for w in perm[g * n:(g + 1) * n]]
+        out[g] = phi[members].astype(np.float64).sum(axis=0) / n
+    return out
 
 
 def outer_step_seeded(phi, theta, delta, seed, step, n, alpha, beta, gamma,

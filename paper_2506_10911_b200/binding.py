@@ -15,13 +15,11 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# NOLO_LIBRARY may name another build of the same library (e.g. one compiled with other tile
-# parameters); by default the library sits next to this file.
-LIB_PATH = os.environ.get("NOLO_LIBRARY") or os.path.join(_HERE, "libnolo.so")
+LIB_PATH = os.path.join(_HERE, "libnolo.so")
 
 NOLO_OK, NOLO_EINVAL, NOLO_ESTATE, NOLO_EALIGN, NOLO_ECUDA, NOLO_ENOMEM = 0, -1, -2, -3, -4, -5
 NOLO_F32, NOLO_BF16 = 0, 1
-NOLO_KERNEL_OUTER, NOLO_KERNEL_ROUTE, NOLO_KERNEL_DIVERGENCE = 0, 1, 2
+NOLO_KERNEL_OUTER, NOLO_KERNEL_ROUTE, NOLO_KERNEL_DIVERGENCE, NOLO_KERNEL_PREPARE = 0, 1, 2, 3
 NOLO_MAX_WORKERS = 4096
 NOLO_STATIC_MAX_WORKERS = 1024
 
@@ -50,6 +48,9 @@ SIGNATURES = {
     "nolo_create": [_i32, _i32, _i64, _i32, _f32, _f32, _f32, ctypes.POINTER(_H)],
     "nolo_bind_state": [_H, _vp, _vp, _vp, _i32, _i64, _vp],
     "nolo_outer_step": [_H, _u64, _u64],
+    "nolo_bind_prepared": [_H, _vp, _i64],
+    "nolo_outer_prepare": [_H, _u64, _u64],
+    "nolo_outer_step_prepared": [_H, _u64, _u64],
     "nolo_outer_step_static": [_i32, _i32, _i64, _f32, _f32, _f32, _vp, _vp, _vp, _i32, _i64, _u64, _u64, _vp,
                                ctypes.c_char_p, _i32],
     "nolo_outer_step_host": [_H, _u64, _u64, _vp, _vp, _vp, _i64],
@@ -65,7 +66,6 @@ SIGNATURES = {
     "nolo_sim_tree_allreduce": [_i32, ctypes.c_double, ctypes.c_double, _i64, _u64, _vp, _vp, _vp],
     "nolo_expected_pair_exchange": [ctypes.c_double, ctypes.c_double],
     "nolo_sim_straggler": [_i32, _i32, _i32, _i32, ctypes.c_double, ctypes.c_double, _i64, _u64, _vp, _vp, _vp],
-    "nolo_device_status": [_H, ctypes.POINTER(ctypes.c_int32)],
     "nolo_timing_enable": [_H, _i32],
     "nolo_timing_read": [_H, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)],
     "nolo_timing_stats": [_H, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)],
@@ -150,6 +150,23 @@ def nolo_outer_step(h: Handle, seed: int, step: int):
     _check(_lib.nolo_outer_step(h.ptr, seed, step), "nolo_outer_step", h)
 
 
+def nolo_bind_prepared(h: Handle, mean_phi, mean_stride=None):
+    """mean_phi: CUDA float64 tensor [W/n, mean_stride] that carries the subgroup means of phi
+    from nolo_outer_prepare to nolo_outer_step_prepared."""
+    if mean_stride is None:
+        mean_stride = mean_phi.stride(0)
+    _check(_lib.nolo_bind_prepared(h.ptr, _ptr(mean_phi), mean_stride), "nolo_bind_prepared", h)
+    h._keep["prepared"] = mean_phi
+
+
+def nolo_outer_prepare(h: Handle, seed: int, next_step: int):
+    _check(_lib.nolo_outer_prepare(h.ptr, seed, next_step), "nolo_outer_prepare", h)
+
+
+def nolo_outer_step_prepared(h: Handle, seed: int, step: int):
+    _check(_lib.nolo_outer_step_prepared(h.ptr, seed, step), "nolo_outer_step_prepared", h)
+
+
 def nolo_outer_step_static(W: int, n: int, P: int, alpha: float, beta: float, gamma: float,
                            phi, theta, delta, seed: int, step: int, stream=None,
                            theta_dtype=None, row_stride=None):
@@ -223,12 +240,6 @@ def nolo_divergence(h: Handle):
     out = (ctypes.c_double * 2)()
     _check(_lib.nolo_divergence(h.ptr, out), "nolo_divergence", h)
     return out[0], out[1]
-
-
-def nolo_device_status(h: Handle) -> int:
-    out = ctypes.c_int32(-1)
-    _check(_lib.nolo_device_status(h.ptr, ctypes.byref(out)), "nolo_device_status", h)
-    return out.value
 
 
 def _stream_ptr(stream):

@@ -12,7 +12,7 @@
 namespace {
 
 constexpr int kMaxTimed = 4096;
-constexpr int kTimedKernels = 3;
+constexpr int kTimedKernels = 4;
 
 struct KernelTimer {
     cudaEvent_t* start = nullptr;
@@ -38,9 +38,14 @@ struct nolo_handle {
     cudaStream_t stream = nullptr;
     bool state_bound = false;
 
-    int32_t* d_perm = nullptr;   // [W], owned
-    int32_t* d_status = nullptr; // 1 word, owned: raised by a kernel whose bounded wait ran out
+    int32_t* d_perm = nullptr;   // [2][W], owned: the table of the last outer step, then that of the last prepare
     bool groups_valid = false;
+
+    // split-phase step: subgroup means of phi prepared ahead of the step (borrowed buffer)
+    double* mean_phi = nullptr;
+    int64_t mean_stride = 0;
+    bool prepared_valid = false;
+    uint64_t prepared_seed = 0, prepared_step = 0;
 
     // routing
     int M = 0, K = 0, act_dtype = NOLO_F32, per_microbatch = 0;
@@ -123,8 +128,12 @@ struct Bracket {
     }
 };
 
-int enqueue_outer(nolo_handle* h, int64_t col0, int64_t cols) {
+int enqueue_outer(nolo_handle* h, int64_t col0, int64_t cols, bool prepared = false) {
     nolo::OuterArgs a;
+    if (prepared) {
+        a.mean_phi = h->mean_phi + col0;
+        a.mean_stride = h->mean_stride;
+    }
     a.phi = h->phi + col0;
     a.theta = static_cast<char*>(h->theta) + col0 * elem_size(h->theta_dtype);
     a.delta = h->delta + col0;
@@ -135,11 +144,11 @@ int enqueue_outer(nolo_handle* h, int64_t col0, int64_t cols) {
     a.n = h->n;
     a.theta_bf16 = h->theta_dtype == NOLO_BF16;
     a.alpha = h->alpha; a.beta = h->beta; a.gamma = h->gamma;
-    a.status = h->d_status;
     Bracket br(h, NOLO_KERNEL_OUTER);
     NOLO_CUDA(h, nolo::launch_outer(a, h->stream));
     br.done();
     ++h->launches;
+    h->prepared_valid = false;   // phi has changed: means prepared from the old phi are stale
     return NOLO_OK;
 }
 
@@ -204,9 +213,7 @@ int nolo_create(int W, int n, int64_t P, int stages, float alpha, float beta, fl
         if (!t.start || !t.stop) { nolo_destroy(h); return NOLO_ENOMEM; }
     }
     cudaError_t e = cudaGetDevice(&h->device);
-    if (e == cudaSuccess) e = cudaMalloc(&h->d_perm, sizeof(int32_t) * (size_t)W);
-    if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(int32_t));
-    if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&h->d_perm, sizeof(int32_t) * 2 * (size_t)W);
     if (e != cudaSuccess) {
         const int code = (e == cudaErrorMemoryAllocation) ? NOLO_ENOMEM : NOLO_ECUDA;
         nolo_destroy(h);
@@ -245,6 +252,56 @@ int nolo_outer_step(nolo_handle* h, uint64_t seed, uint64_t step) {
     int rc = enqueue_group_draw(h, seed, step);
     if (rc != NOLO_OK) return rc;
     return enqueue_outer(h, 0, h->P);
+}
+
+int nolo_bind_prepared(nolo_handle* h, void* mean_phi, int64_t mean_stride) {
+    if (!h) return NOLO_EINVAL;
+    if (!h->state_bound) return fail(h, NOLO_ESTATE, "nolo_bind_state has not been called");
+    if (!mean_phi) return fail(h, NOLO_EINVAL, "mean_phi must not be NULL");
+    if (mean_stride < h->P) return fail(h, NOLO_EINVAL, "mean_stride %lld < P %lld", (long long)mean_stride, (long long)h->P);
+    if (mean_stride % 8 != 0) return fail(h, NOLO_EALIGN, "mean_stride must be a multiple of 8 elements");
+    if (!aligned16(mean_phi)) return fail(h, NOLO_EALIGN, "mean_phi must be 16-byte aligned");
+    const size_t nm = (size_t)(h->W / h->n) * mean_stride * 8;
+    const size_t n4 = (size_t)h->W * h->stride * 4, nt = (size_t)h->W * h->stride * elem_size(h->theta_dtype);
+    if (overlap(mean_phi, nm, h->phi, n4) || overlap(mean_phi, nm, h->delta, n4) || overlap(mean_phi, nm, h->theta, nt))
+        return fail(h, NOLO_EINVAL, "mean_phi overlaps the state");
+    h->mean_phi = static_cast<double*>(mean_phi);
+    h->mean_stride = mean_stride;
+    h->prepared_valid = false;
+    return NOLO_OK;
+}
+
+int nolo_outer_prepare(nolo_handle* h, uint64_t seed, uint64_t next_step) {
+    if (!h) return NOLO_EINVAL;
+    if (!h->state_bound) return fail(h, NOLO_ESTATE, "nolo_bind_state has not been called");
+    if (!h->mean_phi) return fail(h, NOLO_ESTATE, "nolo_bind_prepared has not been called");
+    int32_t* table = h->d_perm + h->W;
+    NOLO_CUDA(h, nolo::launch_draw(seed, next_step, nolo::kDomainGroups, h->W, 1, 1, 1, table, h->stream));
+    ++h->launches;
+    Bracket br(h, NOLO_KERNEL_PREPARE);
+    NOLO_CUDA(h, nolo::launch_group_mean(h->phi, table, h->W, h->n, h->stride, h->P, h->mean_phi, h->mean_stride,
+                                         h->stream));
+    br.done();
+    ++h->launches;
+    h->prepared_valid = true;
+    h->prepared_seed = seed;
+    h->prepared_step = next_step;
+    return NOLO_OK;
+}
+
+int nolo_outer_step_prepared(nolo_handle* h, uint64_t seed, uint64_t step) {
+    if (!h) return NOLO_EINVAL;
+    if (!h->state_bound) return fail(h, NOLO_ESTATE, "nolo_bind_state has not been called");
+    if (!h->mean_phi) return fail(h, NOLO_ESTATE, "nolo_bind_prepared has not been called");
+    if (!h->prepared_valid)
+        return fail(h, NOLO_ESTATE, "no prepared means: call nolo_outer_prepare after the last change of phi");
+    if (h->prepared_seed != seed || h->prepared_step != step)
+        return fail(h, NOLO_ESTATE, "means were prepared for (seed %llu, step %llu), not for (seed %llu, step %llu)",
+                    (unsigned long long)h->prepared_seed, (unsigned long long)h->prepared_step,
+                    (unsigned long long)seed, (unsigned long long)step);
+    int rc = enqueue_group_draw(h, seed, step);
+    if (rc != NOLO_OK) return rc;
+    return enqueue_outer(h, 0, h->P, true);
 }
 
 int nolo_outer_step_host(nolo_handle* h, uint64_t seed, uint64_t step, void* phi_host,
@@ -425,14 +482,6 @@ int nolo_divergence(nolo_handle* h, double* host_out) {
     return NOLO_OK;
 }
 
-int nolo_device_status(nolo_handle* h, int32_t* host_out) {
-    if (!h) return NOLO_EINVAL;
-    if (!host_out) return fail(h, NOLO_EINVAL, "host_out must not be NULL");
-    NOLO_CUDA(h, cudaMemcpyAsync(host_out, h->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, h->stream));
-    NOLO_CUDA(h, cudaStreamSynchronize(h->stream));
-    return NOLO_OK;
-}
-
 int nolo_timing_enable(nolo_handle* h, int enable) {
     if (!h) return NOLO_EINVAL;
     h->timing = enable != 0;
@@ -509,7 +558,6 @@ int nolo_destroy(nolo_handle* h) {
         delete[] t.stop;
     }
     if (h->d_perm) cudaFree(h->d_perm);
-    if (h->d_status) cudaFree(h->d_status);
     if (h->d_route) cudaFree(h->d_route);
     if (h->d_div_partials) cudaFree(h->d_div_partials);
     if (h->d_div_out) cudaFree(h->d_div_out);
@@ -562,6 +610,8 @@ int nolo_sim_straggler(int W, int n, int H, int T, double mu, double sigma, int6
     if (W < 1 || W > NOLO_MAX_WORKERS || n < 1 || n > W || W % n != 0 || H < 1 || T < 1 || trials < 1 ||
         trials > (int64_t(1) << 20) || !std::isfinite(mu) || !std::isfinite(sigma) || sigma < 0 || !host_stats)
         return NOLO_EINVAL;
+    // One launch draws W*H*T samples per trial; a mistyped H or T must not occupy the GPU for hours.
+    if ((double)W * (double)H * (double)T * (double)trials > (double)NOLO_SIM_MAX_SAMPLES) return NOLO_EINVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     double* d = nullptr;
     cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&d), sizeof(double) * (2 * (size_t)trials + 4));

@@ -33,12 +33,20 @@ struct OuterArgs {
     int W, n;
     int theta_bf16;
     float alpha, beta, gamma;
-    int32_t* status = nullptr;  // device word set to 1 if a bounded wait in a kernel ever runs out; may be NULL
+    // Subgroup means of phi prepared in advance (float64, [W/n][mean_stride], row g for subgroup g of
+    // `perm`); NULL = the kernel forms the means itself.
+    const double* mean_phi = nullptr;
+    int64_t mean_stride = 0;
 };
 
 // Fused Eq. 1-3 + theta reset over columns [0, P) of the rows (pointers may be pre-offset by
 // a multiple of 8 columns).  One launch.
 cudaError_t launch_outer(const OuterArgs& a, cudaStream_t stream);
+
+// mean[g][0..P) = float64 mean of phi over subgroup g of `perm` (the part of Eq. 2 that depends on
+// the slow weights only).  One launch.
+cudaError_t launch_group_mean(const float* phi, const int32_t* perm, int W, int n, int64_t stride, int64_t P,
+                              double* mean, int64_t mean_stride, cudaStream_t stream);
 
 struct RouteArgs {
     const void* in;        // [B][R][K][E]

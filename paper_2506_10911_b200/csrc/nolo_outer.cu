@@ -1,80 +1,111 @@
 // Fused NoLoCo outer step (Section 3.2, Eq. 1-3) for W workers resident in one GPU's memory.
 //
 // Work decomposition: one CTA owns one subgroup x one tile of parameters.  Every member's
-// phi / theta / delta element is loaded from HBM exactly once (128-bit coalesced, streaming
+// phi / theta / delta element is fetched from HBM exactly once (128-bit coalesced, streaming
 // cache policy) and every output element stored exactly once; the pseudo-gradients, their sum
-// and the subgroup mean of phi exist only in registers.  The path is bandwidth bound
-// (about 10 flops per 20-24 bytes), so there is no tensor-core work here.
+// and the subgroup mean of phi exist only on chip.  The path is bandwidth bound (about 15 flops
+// per 20-24 bytes), so there is no tensor-core work here.
 //
 //   Delta_j  = phi_j - theta_j                                            (Eq. 1)
 //   delta_i' = alpha*delta_i - (beta/n) sum_j Delta_j - gamma*(phi_i - (1/n) sum_j phi_j)   (Eq. 2)
 //   phi_i'   = phi_i + delta_i'                                           (Eq. 3)
 //   theta_i' = phi_i'   (start of the next inner phase)
+//
+// Three kernels cover the subgroup sizes:
+//   n <= 8        register-resident: one thread holds its quad of every member;
+//   8 < n <= 64   the members are shared out over the warps of one CTA, still in registers;
+//   n > 64        two passes over the members, the second read of phi served by L1/L2.
+//
+// Arithmetic.  Delta_j is formed per member and summed in float32 in short fixed-order partial
+// sums.  gamma * (phi_i - mean phi) is a small number formed from large ones: a mean rounded to
+// float32 would pass half an ulp of |phi| straight into delta', whose tolerance does not grow
+// with |phi|.  So the mean is carried as an unevaluated float32 pair hi + lo (about 46 bits):
+// the register kernel refines a float32 mean by the mean of the residuals phi_j - mean, the
+// other two sum phi with error-free additions (Knuth's two-sum: the rounding error of every
+// addition is recovered exactly and kept in lo).  Float64 accumulators would do the same, but
+// the float32 <-> float64 conversions they need run at 16 per clock per SM on B200 and cost
+// the wide-subgroup kernels 20-35 % of their bandwidth when measured.
 #include "nolo_internal.h"
 
-#include <cooperative_groups.h>
 #include <cuda_bf16.h>
-
-namespace cg = cooperative_groups;
 
 namespace nolo {
 
 namespace {
 
-// Launch shape.  One CTA = kThreads threads; a thread of the register-resident kernel handles
-// ITEMS quads for all members of its subgroup.  The defaults were chosen by measurement on B200.
-#ifndef NOLO_THREADS
-#define NOLO_THREADS 256
-#endif
-#ifndef NOLO_MIN_BLOCKS
-#define NOLO_MIN_BLOCKS 1
-#endif
-#ifndef NOLO_ITEMS_N1
-#define NOLO_ITEMS_N1 4
-#endif
-#ifndef NOLO_ITEMS_N2
-#define NOLO_ITEMS_N2 2
-#endif
-#ifndef NOLO_ITEMS_N4
-#define NOLO_ITEMS_N4 1
-#endif
-#ifndef NOLO_ITEMS_N8
-#define NOLO_ITEMS_N8 1
-#endif
-constexpr int kThreads = NOLO_THREADS;
+constexpr int kThreads = 256;   // CTA size of the register-resident kernel and of the helpers
 
 struct KArgs {
     float* phi;
     void* theta;
     float* delta;
     const int32_t* perm;
+    const double* mean_phi;   // subgroup means of phi prepared in advance, [groups][mean_stride]; or NULL
+    int64_t mean_stride;
     int64_t stride;
     int64_t P;
     int n;
-    float alpha, beta_over_n, gamma, inv_n;
+    float alpha, beta_over_n, gamma, inv_n, n_f;
+    double inv_n_d;
 };
+
+__device__ __forceinline__ void f4_add(float4& s, const float4 v) {
+    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+}
+__device__ __forceinline__ float4 f4_sub(const float4 a, const float4 b) {
+    return make_float4(a.x - b.x, a.y - b.y, a.z - b.z, a.w - b.w);
+}
+__device__ __forceinline__ float4 f4_scale(const float4 a, const float s) {
+    return make_float4(a.x * s, a.y * s, a.z * s, a.w * s);
+}
+__device__ __forceinline__ float4 f4_zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+
+// ---- the mean of phi as a float32 pair ----------------------------------------------------
+
+// hi + x with the rounding error of the addition added to lo (error-free: hi_new + error == hi + x).
+__device__ __forceinline__ void two_sum(float& hi, float& lo, const float x) {
+    const float s = hi + x;
+    const float bb = s - hi;
+    lo += (hi - (s - bb)) + (x - bb);
+    hi = s;
+}
+
+// Running sum of the phi quads of some members, later the mean: value = hi + lo.
+struct PairSum {
+    float4 hi, lo;
+    __device__ __forceinline__ void clear() { hi = f4_zero(); lo = f4_zero(); }
+    __device__ __forceinline__ void add(const float4 v) {
+        two_sum(hi.x, lo.x, v.x); two_sum(hi.y, lo.y, v.y); two_sum(hi.z, lo.z, v.z); two_sum(hi.w, lo.w, v.w);
+    }
+    __device__ __forceinline__ void add(const PairSum& o) { add(o.hi); f4_add(lo, o.lo); }
+    // sum -> sum / n.  m = fl(hi / n) leaves hi - m*n, which the fused multiply-add returns exactly.
+    static __device__ __forceinline__ void divide1(float& h, float& l, const float inv_n, const float n_f) {
+        const float m = h * inv_n;
+        const float r = fmaf(-m, n_f, h);
+        l = (r + l) * inv_n;
+        h = m;
+    }
+    __device__ __forceinline__ void divide(const KArgs& a) {
+        divide1(hi.x, lo.x, a.inv_n, a.n_f); divide1(hi.y, lo.y, a.inv_n, a.n_f);
+        divide1(hi.z, lo.z, a.inv_n, a.n_f); divide1(hi.w, lo.w, a.inv_n, a.n_f);
+    }
+    // phi - mean
+    __device__ __forceinline__ float4 deviation(const float4 phi) const { return f4_sub(f4_sub(phi, hi), lo); }
+};
+
+// The mean of subgroup g for quad q prepared in advance (float64 in memory), split into hi + lo.
+__device__ __forceinline__ PairSum load_prepared_mean(const KArgs& a, int g, int64_t q) {
+    const double2* m = reinterpret_cast<const double2*>(a.mean_phi + (int64_t)g * a.mean_stride) + 2 * q;
+    const double2 u = __ldg(m), v = __ldg(m + 1);
+    PairSum p;
+    p.hi = make_float4((float)u.x, (float)u.y, (float)v.x, (float)v.y);
+    p.lo = make_float4((float)(u.x - (double)p.hi.x), (float)(u.y - (double)p.hi.y),
+                       (float)(v.x - (double)p.hi.z), (float)(v.y - (double)p.hi.w));
+    return p;
+}
 
 // ---- theta access: 4 consecutive parameters as float4, fp32 or bf16 storage -------------
 
-__device__ __forceinline__ float4 load_theta4(const float* row, int64_t q) {
-    return __ldcs(reinterpret_cast<const float4*>(row) + q);
-}
-__device__ __forceinline__ float4 load_theta4(const __nv_bfloat16* row, int64_t q) {
-    const uint2 v = __ldcs(reinterpret_cast<const uint2*>(row) + q);
-    float4 r;
-    r.x = __uint_as_float(v.x << 16);
-    r.y = __uint_as_float(v.x & 0xffff0000u);
-    r.z = __uint_as_float(v.y << 16);
-    r.w = __uint_as_float(v.y & 0xffff0000u);
-    return r;
-}
-// Raw (unconverted) loads, so that the conversion sits with the arithmetic and never between loads.
-__device__ __forceinline__ float4 load_theta_raw(const float* row, int64_t q) {
-    return __ldcs(reinterpret_cast<const float4*>(row) + q);
-}
-__device__ __forceinline__ uint2 load_theta_raw(const __nv_bfloat16* row, int64_t q) {
-    return __ldcs(reinterpret_cast<const uint2*>(row) + q);
-}
 __device__ __forceinline__ float4 widen(float4 v) { return v; }
 __device__ __forceinline__ float4 widen(uint2 v) {
     float4 r;
@@ -83,6 +114,14 @@ __device__ __forceinline__ float4 widen(uint2 v) {
     r.z = __uint_as_float(v.y << 16);
     r.w = __uint_as_float(v.y & 0xffff0000u);
     return r;
+}
+// Raw (unconverted) loads, so that the conversion sits with the arithmetic and never between loads
+// (a conversion placed between the loads serialised them when measured).
+__device__ __forceinline__ float4 load_theta_raw(const float* row, int64_t q) {
+    return __ldcs(reinterpret_cast<const float4*>(row) + q);
+}
+__device__ __forceinline__ uint2 load_theta_raw(const __nv_bfloat16* row, int64_t q) {
+    return __ldcs(reinterpret_cast<const uint2*>(row) + q);
 }
 template <typename ThetaT> struct ThetaRaw { using type = float4; };
 template <> struct ThetaRaw<__nv_bfloat16> { using type = uint2; };
@@ -107,31 +146,52 @@ __device__ __forceinline__ void store_theta1(__nv_bfloat16* row, int64_t c, floa
     row[c] = __float2bfloat16_rn(v);
 }
 
-__device__ __forceinline__ float update1(float phi, float delta, float sum_Delta, float mean_phi,
+// Eq. 2 and Eq. 3 for one parameter; dev = phi_i - mean phi.
+__device__ __forceinline__ float update1(float phi, float dev, float delta, float sum_Delta,
                                          const KArgs& a, float* delta_out) {
-    const float d = a.alpha * delta - a.beta_over_n * sum_Delta - a.gamma * (phi - mean_phi);
+    const float d = a.alpha * delta - a.beta_over_n * sum_Delta - a.gamma * dev;
     *delta_out = d;
     return phi + d;
 }
+__device__ __forceinline__ float4 update4(const float4 phi, const float4 dev, const float4 delta,
+                                          const float4 sum_Delta, const KArgs& a, float4* delta_out) {
+    float4 p;
+    p.x = update1(phi.x, dev.x, delta.x, sum_Delta.x, a, &delta_out->x);
+    p.y = update1(phi.y, dev.y, delta.y, sum_Delta.y, a, &delta_out->y);
+    p.z = update1(phi.z, dev.z, delta.z, sum_Delta.z, a, &delta_out->z);
+    p.w = update1(phi.w, dev.w, delta.w, sum_Delta.w, a, &delta_out->w);
+    return p;
+}
+// update and store one member's quad
+template <typename ThetaT>
+__device__ __forceinline__ void update_store(const KArgs& a, int64_t row_off, int64_t q, const float4 phi,
+                                             const float4 dev, const float4 delta, const float4 sum_Delta) {
+    float4 d;
+    const float4 p = update4(phi, dev, delta, sum_Delta, a, &d);
+    __stcs(reinterpret_cast<float4*>(a.phi + row_off) + q, p);
+    __stcs(reinterpret_cast<float4*>(a.delta + row_off) + q, d);
+    store_theta4(static_cast<ThetaT*>(a.theta) + row_off, q, p);
+}
 
-// Columns P - (P % 4) .. P-1 of one subgroup, element by element (rows are only guaranteed to be
-// padded to a multiple of 8, and padding must not be written).
+// Columns P - (P % 4) .. P-1 of one subgroup, element by element in float64 (rows are only
+// guaranteed to be padded to a multiple of 8, and padding must not be written).
 template <typename ThetaT>
 __device__ void scalar_tail(const KArgs& a, int g) {
     const int n = a.n;
     for (int64_t c = a.P & ~int64_t(3); c < a.P; ++c) {
-        float sD = 0.f, sP = 0.f;
+        double sD = 0.0, sP = 0.0;
         for (int j = 0; j < n; ++j) {
             const int64_t row = (int64_t)a.perm[g * n + j] * a.stride;
             const float p = a.phi[row + c];
-            sD += p - load_theta1(static_cast<const ThetaT*>(a.theta) + row, c);
-            sP += p;
+            sD += (double)(p - load_theta1(static_cast<const ThetaT*>(a.theta) + row, c));
+            sP += (double)p;
         }
-        const float mP = sP * a.inv_n;
+        const double mP = a.mean_phi ? a.mean_phi[(int64_t)g * a.mean_stride + c] : sP * a.inv_n_d;
         for (int j = 0; j < n; ++j) {
             const int64_t row = (int64_t)a.perm[g * n + j] * a.stride;
             float d;
-            const float p = update1(a.phi[row + c], a.delta[row + c], sD, mP, a, &d);
+            const float p0 = a.phi[row + c];
+            const float p = update1(p0, (float)((double)p0 - mP), a.delta[row + c], (float)sD, a, &d);
             a.phi[row + c] = p;
             a.delta[row + c] = d;
             store_theta1(static_cast<ThetaT*>(a.theta) + row, c, p);
@@ -139,13 +199,14 @@ __device__ void scalar_tail(const KArgs& a, int g) {
     }
 }
 
-// ---- register-resident path: subgroup size N known at compile time ----------------------
+// ---- n <= 8: register-resident, subgroup size N known at compile time --------------------
 //
 // Each thread handles ITEMS quads (4 consecutive parameters) of the tile, 256 quads apart, for all
 // N members: phi_j stays in registers between the reduction and the update, so nothing is read
 // twice.  All loads of a thread are issued before the first use to keep many bytes in flight.
-template <int N, typename ThetaT, int ITEMS>
-__global__ void __launch_bounds__(kThreads, NOLO_MIN_BLOCKS)
+// ITEMS = 4 for n = 1, 2 for pairs with float32 theta, 1 otherwise (chosen by measurement).
+template <int N, typename ThetaT, int ITEMS, bool PREPARED>
+__global__ void __launch_bounds__(kThreads, 1)
 outer_step_reg_kernel(const KArgs a) {
     const int g = blockIdx.y;
     const int64_t full_quads = a.P >> 2;
@@ -158,7 +219,8 @@ outer_step_reg_kernel(const KArgs a) {
     auto delta_row = [&](int j) { return a.delta + (int64_t)row[j] * a.stride; };
     auto theta_row = [&](int j) { return static_cast<ThetaT*>(a.theta) + (int64_t)row[j] * a.stride; };
 
-    float4 phi[ITEMS][N], dlt[ITEMS][N], the[ITEMS][N];
+    float4 phi[ITEMS][N], dlt[ITEMS][N];
+    typename ThetaRaw<ThetaT>::type the[ITEMS][N];
     bool ok[ITEMS];
 #pragma unroll
     for (int it = 0; it < ITEMS; ++it) {
@@ -168,7 +230,7 @@ outer_step_reg_kernel(const KArgs a) {
 #pragma unroll
             for (int j = 0; j < N; ++j) {
                 phi[it][j] = __ldcs(reinterpret_cast<const float4*>(phi_row(j)) + q);
-                the[it][j] = load_theta4(theta_row(j), q);
+                the[it][j] = load_theta_raw(theta_row(j), q);
             }
 #pragma unroll
             for (int j = 0; j < N; ++j)
@@ -179,89 +241,75 @@ outer_step_reg_kernel(const KArgs a) {
     for (int it = 0; it < ITEMS; ++it) {
         if (!ok[it]) continue;
         const int64_t q = q0 + (int64_t)it * kThreads;
-        float4 sD = make_float4(0.f, 0.f, 0.f, 0.f), sP = sD;
-#pragma unroll
-        for (int j = 0; j < N; ++j) {          // fixed member order: deterministic sums
-            sD.x += phi[it][j].x - the[it][j].x;  sP.x += phi[it][j].x;
-            sD.y += phi[it][j].y - the[it][j].y;  sP.y += phi[it][j].y;
-            sD.z += phi[it][j].z - the[it][j].z;  sP.z += phi[it][j].z;
-            sD.w += phi[it][j].w - the[it][j].w;  sP.w += phi[it][j].w;
-        }
-        const float4 mP = make_float4(sP.x * a.inv_n, sP.y * a.inv_n, sP.z * a.inv_n, sP.w * a.inv_n);
+        // Sums in the fixed member order (deterministic).  The mean of phi is formed in two
+        // passes over the registers: a plain float32 mean, then the mean of the residuals
+        // phi_j - mean, so that hi + lo keeps the precision of the spread of the replicas.
+        float4 sD = f4_zero(), s0 = f4_zero();
 #pragma unroll
         for (int j = 0; j < N; ++j) {
-            float4 d, p;
-            p.x = update1(phi[it][j].x, dlt[it][j].x, sD.x, mP.x, a, &d.x);
-            p.y = update1(phi[it][j].y, dlt[it][j].y, sD.y, mP.y, a, &d.y);
-            p.z = update1(phi[it][j].z, dlt[it][j].z, sD.z, mP.z, a, &d.z);
-            p.w = update1(phi[it][j].w, dlt[it][j].w, sD.w, mP.w, a, &d.w);
-            __stcs(reinterpret_cast<float4*>(phi_row(j)) + q, p);
-            __stcs(reinterpret_cast<float4*>(delta_row(j)) + q, d);
-            store_theta4(theta_row(j), q, p);
+            f4_add(sD, f4_sub(phi[it][j], widen(the[it][j])));          // Eq. 1
+            f4_add(s0, phi[it][j]);
         }
+        PairSum mean;
+        if (PREPARED) {
+            mean = load_prepared_mean(a, g, q);
+        } else {
+            mean.hi = f4_scale(s0, a.inv_n);
+            float4 sR = f4_zero();
+#pragma unroll
+            for (int j = 0; j < N; ++j) f4_add(sR, f4_sub(phi[it][j], mean.hi));
+            mean.lo = f4_scale(sR, a.inv_n);
+        }
+#pragma unroll
+        for (int j = 0; j < N; ++j)
+            update_store<ThetaT>(a, (int64_t)row[j] * a.stride, q, phi[it][j], mean.deviation(phi[it][j]),
+                                 dlt[it][j], sD);
     }
     if ((a.P & 3) && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) scalar_tail<ThetaT>(a, g);
 }
 
-// ---- large subgroups (8 < n <= 64, 192 < n <= 256): members split across warps, CTAs and a cluster
+// ---- 8 < n <= 64: the members shared out over the warps of one CTA ------------------------
 //
 // Holding phi of every member of a tile in registers costs n x 512 bytes per 32 quads, and the
 // kernel only streams at full bandwidth while more than one CTA fits on an SM (one CTA's loads
-// must overlap another's barrier and stores).  So a CTA takes at most 64 members: warp w of its
-// G <= 8 warps holds up to 8 members, w*MPW .. w*MPW+MPW-1 of the CTA's share, for the same 32
-// quads (each member row is read in coalesced 512-byte segments), and a larger subgroup is spread
-// over a thread-block cluster of C = 2 or 4 CTAs that work on the same tile.  Partial sums meet
-// in shared memory (warps of a CTA) and then in distributed shared memory (CTAs of the cluster);
-// both are added in a fixed order, so the result is deterministic and identical in every CTA.
-// As in the small-n kernel every element is read once and written once.  The CTA shape (64
-// members, 8 per warp) measured best on B200 among 32/64/128 members and 4/8 per warp.
-#ifndef NOLO_SPLIT_CTA_MEMBERS
-#define NOLO_SPLIT_CTA_MEMBERS 64     // members one CTA holds (larger subgroups use a cluster)
-#endif
-#ifndef NOLO_SPLIT_PREF
-#define NOLO_SPLIT_PREF 8             // members per warp aimed at when a CTA has more than 16 members
-#endif
-constexpr int kSplitMaxCluster = 4;    // larger clusters measured slower than the two-pass kernel
-constexpr int kSplitMembersPerCta = NOLO_SPLIT_CTA_MEMBERS;
-constexpr int kSplitMaxWarps = 16;
+// must overlap another's barrier and stores).  Warp w of the G <= 8 warps holds up to 8 members,
+// w*MPW .. w*MPW+MPW-1, for the same 32 quads (each member row is read in coalesced 512-byte
+// segments); the warps' partial sums meet in shared memory and are added in warp order, so the
+// result is deterministic and identical in every warp.  As in the small-n kernel every element
+// is read once and written once.  The shape (8 members per warp) measured best on B200 among
+// 4 and 8 per warp and CTAs of 32 / 64 / 128 members.
+constexpr int kSplitMaxMembers = 64;   // members one CTA holds
+constexpr int kSplitPref = 8;          // members per warp aimed at when the subgroup has more than 16 members
+constexpr int kSplitMaxWarps = kSplitMaxMembers / kSplitPref;
 
-// Launch bounds: MAXW warps per CTA; registers per thread capped so that several CTAs fit an SM.
-template <int MPW, int MAXW>
+// Registers per thread capped so that several CTAs fit an SM.
+template <int MPW>
 struct SplitShape {
     static constexpr int kRegs = MPW <= 4 ? 80 : 128;
-    static constexpr int kMinBlocks = (65536 / (MAXW * 32 * kRegs)) > 0 ? (65536 / (MAXW * 32 * kRegs)) : 1;
+    static constexpr int kMinBlocks = 65536 / (kSplitMaxWarps * 32 * kRegs);
 };
 
-template <int MPW, typename ThetaT, bool CLUSTER, int MAXW>
-__global__ void __launch_bounds__(MAXW * 32, SplitShape<MPW, MAXW>::kMinBlocks)
-outer_step_split_kernel(const KArgs a, int members_per_cta) {
-    __shared__ float4 part_D[MAXW][32];
-    __shared__ float4 part_P[MAXW][32];
-    __shared__ float4 cta_D[32];
-    __shared__ float4 cta_P[32];
+template <int MPW, typename ThetaT>
+__global__ void __launch_bounds__(kSplitMaxWarps * 32, SplitShape<MPW>::kMinBlocks)
+outer_step_split_kernel(const KArgs a) {
+    __shared__ float4 part_D[kSplitMaxWarps][32];
+    __shared__ PairSum part_P[kSplitMaxWarps][32];
     const int G = blockDim.x >> 5;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = blockIdx.y;
     const int n = a.n;
-    int C = 1, rank = 0;
-    if (CLUSTER) {
-        cg::cluster_group cluster = cg::this_cluster();
-        C = (int)cluster.num_blocks();
-        rank = (int)cluster.block_rank();
-    }
-    const int64_t tile = CLUSTER ? (int64_t)(blockIdx.x / C) : (int64_t)blockIdx.x;
-    const int64_t q = tile * 32 + lane;
+    const int64_t q = (int64_t)blockIdx.x * 32 + lane;
     const bool ok = q < (a.P >> 2);
-    const int j_begin = rank * members_per_cta;
-    const int j_end = min(n, j_begin + members_per_cta);
-    const int j0 = j_begin + warp * MPW;
+    const int j0 = warp * MPW;
 
     int row[MPW];
 #pragma unroll
-    for (int m = 0; m < MPW; ++m) row[m] = (j0 + m < j_end) ? __ldg(a.perm + g * n + j0 + m) : -1;
+    for (int m = 0; m < MPW; ++m) row[m] = (j0 + m < n) ? __ldg(a.perm + g * n + j0 + m) : -1;
 
     float4 phi[MPW], dlt[MPW];
-    float4 sD = make_float4(0.f, 0.f, 0.f, 0.f), sP = sD;
+    float4 sD = f4_zero();
+    PairSum sP;
+    sP.clear();
     if (ok) {
         typename ThetaRaw<ThetaT>::type raw[MPW];
 #pragma unroll
@@ -280,383 +328,287 @@ outer_step_split_kernel(const KArgs a, int members_per_cta) {
 #pragma unroll
         for (int m = 0; m < MPW; ++m) {
             if (row[m] >= 0) {
-                const float4 t = widen(raw[m]);
-                sD.x += phi[m].x - t.x;  sP.x += phi[m].x;
-                sD.y += phi[m].y - t.y;  sP.y += phi[m].y;
-                sD.z += phi[m].z - t.z;  sP.z += phi[m].z;
-                sD.w += phi[m].w - t.w;  sP.w += phi[m].w;
+                f4_add(sD, f4_sub(phi[m], widen(raw[m])));          // Eq. 1
+                sP.add(phi[m]);
             }
         }
     }
     part_D[warp][lane] = sD;
     part_P[warp][lane] = sP;
     __syncthreads();
-    // sum over the warps of this CTA, in warp order
-    sD = part_D[0][lane];
-    sP = part_P[0][lane];
-    for (int w = 1; w < G; ++w) {
-        const float4 d = part_D[w][lane], p = part_P[w][lane];
-        sD.x += d.x; sD.y += d.y; sD.z += d.z; sD.w += d.w;
-        sP.x += p.x; sP.y += p.y; sP.z += p.z; sP.w += p.w;
-    }
-    if (CLUSTER) {
-        cg::cluster_group cluster = cg::this_cluster();
-        if (warp == 0) {
-            cta_D[lane] = sD;
-            cta_P[lane] = sP;
-        }
-        cluster.sync();                       // every CTA's sums are published
-        // sum over the CTAs of the cluster, in rank order, through distributed shared memory
-        const float4* rD = cluster.map_shared_rank(cta_D, 0);
-        const float4* rP = cluster.map_shared_rank(cta_P, 0);
-        sD = rD[lane];
-        sP = rP[lane];
-        for (int c = 1; c < C; ++c) {
-            rD = cluster.map_shared_rank(cta_D, c);
-            rP = cluster.map_shared_rank(cta_P, c);
-            const float4 d = rD[lane], p = rP[lane];
-            sD.x += d.x; sD.y += d.y; sD.z += d.z; sD.w += d.w;
-            sP.x += p.x; sP.y += p.y; sP.z += p.z; sP.w += p.w;
-        }
-        cluster.barrier_arrive();             // this CTA no longer reads its peers' shared memory
-    }
     if (ok) {
-        const float4 mP = make_float4(sP.x * a.inv_n, sP.y * a.inv_n, sP.z * a.inv_n, sP.w * a.inv_n);
+        // sum over the warps of this CTA, in warp order
+        sD = part_D[0][lane];
+        sP = part_P[0][lane];
+        for (int w = 1; w < G; ++w) {
+            f4_add(sD, part_D[w][lane]);
+            sP.add(part_P[w][lane]);
+        }
+        if (a.mean_phi) sP = load_prepared_mean(a, g, q);
+        else sP.divide(a);
 #pragma unroll
         for (int m = 0; m < MPW; ++m) {
-            if (row[m] >= 0) {
-                const int64_t off = (int64_t)row[m] * a.stride;
-                float4 d, p;
-                p.x = update1(phi[m].x, dlt[m].x, sD.x, mP.x, a, &d.x);
-                p.y = update1(phi[m].y, dlt[m].y, sD.y, mP.y, a, &d.y);
-                p.z = update1(phi[m].z, dlt[m].z, sD.z, mP.z, a, &d.z);
-                p.w = update1(phi[m].w, dlt[m].w, sD.w, mP.w, a, &d.w);
-                __stcs(reinterpret_cast<float4*>(a.phi + off) + q, p);
-                __stcs(reinterpret_cast<float4*>(a.delta + off) + q, d);
-                store_theta4(static_cast<ThetaT*>(a.theta) + off, q, p);
+            if (row[m] >= 0)
+                update_store<ThetaT>(a, (int64_t)row[m] * a.stride, q, phi[m], sP.deviation(phi[m]), dlt[m], sD);
+        }
+    }
+    if ((a.P & 3) && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) scalar_tail<ThetaT>(a, g);
+}
+
+// ---- n > 64: two passes over the members, the second read of phi served by L1 / L2 ---------
+//
+// One CTA owns one subgroup x ROWQ quads.  Its threads form WARPS*32/ROWQ slots of ROWQ lanes;
+// slot s walks members s, s + SLOTS, ... in chunks of U rows in flight.  Pass 1 reads phi and
+// theta and accumulates the two sums; the slots' partial sums meet in shared memory; pass 2
+// reads phi again together with delta and writes the update.  Between the two reads of a phi
+// element lie only the other rows of the same CTA's tile (n x ROWQ x 16 bytes, 32-128 KB for the
+// shapes used), so the second read is served by L1 or L2: profiled DRAM traffic equals the
+// algorithmic 24 / 20 bytes per worker-parameter, and nothing has to be parked in registers or
+// shared memory, whatever n is.  No bulk copies, no clusters and no waits other than the one CTA
+// barrier.  Shapes (by measurement): 8 warps x 32 quads x 4 rows in flight, 3 CTAs per SM, up to
+// 320 members; 16 warps x 16 quads x 8 rows above (narrower segments keep the tile cacheable).
+template <typename ThetaT, int WARPS, int ROWQ, int U, int MINB>
+__global__ void __launch_bounds__(WARPS * 32, MINB)
+outer_step_twopass_kernel(const KArgs a) {
+    constexpr int SLOTS = WARPS * 32 / ROWQ;
+    constexpr int SPW = 32 / ROWQ;            // slots per warp
+    static_assert(ROWQ == 32 || ROWQ == 16 || ROWQ == 8, "a slot is a whole fraction of a warp");
+    __shared__ float4 part_D[WARPS][ROWQ];
+    __shared__ PairSum part_P[WARPS][ROWQ];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ql = lane % ROWQ;
+    const int slot = warp * SPW + lane / ROWQ;
+    const int g = blockIdx.y;
+    const int n = a.n;
+    const int32_t* members = a.perm + (int64_t)g * n;
+    const int64_t q = (int64_t)blockIdx.x * ROWQ + ql;
+    const bool ok = q < (a.P >> 2);
+
+    float4 sD = f4_zero();
+    PairSum sP;
+    sP.clear();
+    if (ok) {
+        for (int j = slot; j < n; j += SLOTS * U) {
+            float4 p[U];
+            typename ThetaRaw<ThetaT>::type t[U];
+#pragma unroll
+            for (int i = 0; i < U; ++i) {
+                const int jj = j + i * SLOTS;
+                if (jj < n) {
+                    const int64_t off = (int64_t)__ldg(members + jj) * a.stride;
+                    p[i] = reinterpret_cast<const float4*>(a.phi + off)[q];     // default policy: stays cached for pass 2
+                    t[i] = load_theta_raw(static_cast<const ThetaT*>(a.theta) + off, q);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < U; ++i) {
+                if (j + i * SLOTS < n) {
+                    f4_add(sD, f4_sub(p[i], widen(t[i])));              // Eq. 1
+                    sP.add(p[i]);
+                }
             }
         }
     }
-    if ((a.P & 3) && rank == 0 && tile == (int64_t)(gridDim.x / C) - 1 && threadIdx.x == 0)
-        scalar_tail<ThetaT>(a, g);
-    if (CLUSTER) cg::this_cluster().barrier_wait();   // peers may still be reading this CTA's sums
-}
-
-// ---- 64 < n <= 192: phi staged in shared memory by bulk-async copies ------------------------
-//
-// One CTA of 8 warps (16 above 112 members) owns one subgroup x 32 quads, for all n members.  The members' phi segments
-// (512 bytes each) are brought into shared memory by cp.async.bulk copies that complete on one
-// mbarrier, so phi needs no registers while it waits for the reduction; meanwhile every warp
-// streams the theta segments of its own members through registers and sums them.  After the
-// mbarrier and one CTA barrier each warp updates its own members: phi from shared memory, delta
-// from global memory.  sum_Delta is formed as sum(phi) - sum(theta), both in a fixed order.
-// Still one read and one write per element; n x 512 bytes of shared memory per CTA, 3 CTAs per SM
-// at n = 128, 2 at n = 192.  Measured 2 to 19 % faster than spreading such a subgroup over a cluster
-// of CTAs; from about 256 members on the cluster kernel below is the faster one again.
-// The wait on the mbarrier is bounded: if it ever ran out, the CTA would leave its
-// tile untouched and raise the status word instead of hanging.
-#ifndef NOLO_STAGED
-#define NOLO_STAGED 1
-#endif
-#ifndef NOLO_STAGED_MAX_N
-#define NOLO_STAGED_MAX_N 192
-#endif
-#ifndef NOLO_STAGED_SPLIT
-#define NOLO_STAGED_SPLIT 112      // up to here 8 warps, above 16 (8 to 14 members per warp)
-#endif
-constexpr int kStagedChunk = 4;      // member rows in flight per thread
-constexpr int kStagedWaitLimit = 1 << 20;
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-
-template <typename ThetaT, int kStagedWarps>
-__global__ void __launch_bounds__(kStagedWarps * 32, kStagedWarps <= 8 ? 3 : 2)
-outer_step_staged_kernel(const KArgs a, int32_t* __restrict__ status) {
-    extern __shared__ __align__(128) unsigned char staged_smem[];
-    float4* phi_s = reinterpret_cast<float4*>(staged_smem);          // [n][32] quads
-    __shared__ float4 part_T[kStagedWarps][32];
-    __shared__ float4 part_P[kStagedWarps][32];
-    __shared__ __align__(8) uint64_t bar;
-    __shared__ int timed_out;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = blockIdx.y;
-    const int n = a.n;
-    const int32_t* members = a.perm + (int64_t)g * n;
-    const int64_t full_quads = a.P >> 2;
-    const int64_t q0 = (int64_t)blockIdx.x * 32;
-    const int tile_quads = (int)(full_quads - q0 < 32 ? (full_quads - q0 > 0 ? full_quads - q0 : 0) : 32);
-    const uint32_t row_bytes = (uint32_t)tile_quads * 16u;
-    const uint32_t bar_addr = smem_u32(&bar);
-
-    if (threadIdx.x == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_addr) : "memory");
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        timed_out = 0;
+    // the slots of one warp that share a quad (fixed order), then the warps through shared memory
+#pragma unroll
+    for (int o = ROWQ; o < 32; o <<= 1) {
+        PairSum t;
+        float4 d;
+        d.x = __shfl_xor_sync(0xffffffffu, sD.x, o); d.y = __shfl_xor_sync(0xffffffffu, sD.y, o);
+        d.z = __shfl_xor_sync(0xffffffffu, sD.z, o); d.w = __shfl_xor_sync(0xffffffffu, sD.w, o);
+        t.hi.x = __shfl_xor_sync(0xffffffffu, sP.hi.x, o); t.hi.y = __shfl_xor_sync(0xffffffffu, sP.hi.y, o);
+        t.hi.z = __shfl_xor_sync(0xffffffffu, sP.hi.z, o); t.hi.w = __shfl_xor_sync(0xffffffffu, sP.hi.w, o);
+        t.lo.x = __shfl_xor_sync(0xffffffffu, sP.lo.x, o); t.lo.y = __shfl_xor_sync(0xffffffffu, sP.lo.y, o);
+        t.lo.z = __shfl_xor_sync(0xffffffffu, sP.lo.z, o); t.lo.w = __shfl_xor_sync(0xffffffffu, sP.lo.w, o);
+        // both partners add (lower slot) + (higher slot) in that order, so they agree bit for bit
+        if (lane & o) {
+            PairSum mine = sP;
+            sP = t;
+            sP.add(mine);
+            d.x += sD.x; d.y += sD.y; d.z += sD.z; d.w += sD.w;
+            sD = d;
+        } else {
+            sP.add(t);
+            f4_add(sD, d);
+        }
+    }
+    if (lane < ROWQ) {
+        part_D[warp][ql] = sD;
+        part_P[warp][ql] = sP;
     }
     __syncthreads();
-    if (warp == 0 && tile_quads > 0) {
-        if (lane == 0)
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr),
-                         "r"((uint32_t)n * row_bytes)
-                         : "memory");
-        __syncwarp();
-        for (int j = lane; j < n; j += 32) {
-            const float* src = a.phi + (int64_t)__ldg(members + j) * a.stride + q0 * 4;
-            asm volatile(
-                "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                    smem_u32(phi_s + (size_t)j * 32)),
-                "l"(src), "r"(row_bytes), "r"(bar_addr)
-                : "memory");
-        }
-    }
-
-    // theta of this warp's members, through registers
-    const int mpw = (n + kStagedWarps - 1) / kStagedWarps;
-    const int j_begin = warp * mpw;
-    const int j_end = min(n, j_begin + mpw);
-    const bool ok = lane < tile_quads;
-    const int64_t q = q0 + lane;
-    float4 sT = make_float4(0.f, 0.f, 0.f, 0.f), sP = sT;
     if (ok) {
-        for (int j = j_begin; j < j_end; j += kStagedChunk) {
-            typename ThetaRaw<ThetaT>::type raw[kStagedChunk];
+        sD = part_D[0][ql];
+        sP = part_P[0][ql];
 #pragma unroll
-            for (int i = 0; i < kStagedChunk; ++i)
-                if (j + i < j_end)
-                    raw[i] = load_theta_raw(
-                        static_cast<const ThetaT*>(a.theta) + (int64_t)__ldg(members + j + i) * a.stride, q);
+        for (int w = 1; w < WARPS; ++w) {
+            f4_add(sD, part_D[w][ql]);
+            sP.add(part_P[w][ql]);
+        }
+        if (a.mean_phi) sP = load_prepared_mean(a, g, q);
+        else sP.divide(a);
+        for (int j = slot; j < n; j += SLOTS * U) {
+            float4 p[U], dl[U];
+            int64_t off[U];
 #pragma unroll
-            for (int i = 0; i < kStagedChunk; ++i)
-                if (j + i < j_end) {
-                    const float4 t = widen(raw[i]);
-                    sT.x += t.x; sT.y += t.y; sT.z += t.z; sT.w += t.w;
-                }
-        }
-    }
-    if (tile_quads > 0) {                     // bounded wait for the phi segments
-        bool done = false;
-        for (int it = 0; it < kStagedWaitLimit && !done; ++it) {
-            uint32_t ready;
-            asm volatile(
-                "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n selp.u32 %0, 1, 0, p;\n}\n"
-                : "=r"(ready)
-                : "r"(bar_addr)
-                : "memory");
-            done = ready != 0;
-        }
-        if (!done) timed_out = 1;
-    }
-    if (ok && !timed_out) {
-        for (int j = j_begin; j < j_end; ++j) {
-            const float4 p = phi_s[(size_t)j * 32 + lane];
-            sP.x += p.x; sP.y += p.y; sP.z += p.z; sP.w += p.w;
-        }
-    }
-    part_T[warp][lane] = sT;
-    part_P[warp][lane] = sP;
-    __syncthreads();
-    if (timed_out) {                           // same value in every thread after the barrier
-        if (threadIdx.x == 0 && status) atomicExch(status, 1);
-        return;
-    }
-    if (ok) {
-        float4 tT = part_T[0][lane], tP = part_P[0][lane];
-#pragma unroll
-        for (int w = 1; w < kStagedWarps; ++w) {
-            const float4 t = part_T[w][lane], p = part_P[w][lane];
-            tT.x += t.x; tT.y += t.y; tT.z += t.z; tT.w += t.w;
-            tP.x += p.x; tP.y += p.y; tP.z += p.z; tP.w += p.w;
-        }
-        const float4 sD = make_float4(tP.x - tT.x, tP.y - tT.y, tP.z - tT.z, tP.w - tT.w);
-        const float4 mP = make_float4(tP.x * a.inv_n, tP.y * a.inv_n, tP.z * a.inv_n, tP.w * a.inv_n);
-        for (int j = j_begin; j < j_end; j += kStagedChunk) {
-            float4 dl[kStagedChunk];
-            int64_t off[kStagedChunk];
-#pragma unroll
-            for (int i = 0; i < kStagedChunk; ++i)
-                if (j + i < j_end) {
-                    off[i] = (int64_t)__ldg(members + j + i) * a.stride;
+            for (int i = 0; i < U; ++i) {
+                const int jj = j + i * SLOTS;
+                if (jj < n) {
+                    off[i] = (int64_t)__ldg(members + jj) * a.stride;
+                    p[i] = __ldcs(reinterpret_cast<const float4*>(a.phi + off[i]) + q);
                     dl[i] = __ldcs(reinterpret_cast<const float4*>(a.delta + off[i]) + q);
                 }
+            }
 #pragma unroll
-            for (int i = 0; i < kStagedChunk; ++i)
-                if (j + i < j_end) {
-                    const float4 p0 = phi_s[(size_t)(j + i) * 32 + lane];
-                    float4 d, p;
-                    p.x = update1(p0.x, dl[i].x, sD.x, mP.x, a, &d.x);
-                    p.y = update1(p0.y, dl[i].y, sD.y, mP.y, a, &d.y);
-                    p.z = update1(p0.z, dl[i].z, sD.z, mP.z, a, &d.z);
-                    p.w = update1(p0.w, dl[i].w, sD.w, mP.w, a, &d.w);
-                    __stcs(reinterpret_cast<float4*>(a.phi + off[i]) + q, p);
-                    __stcs(reinterpret_cast<float4*>(a.delta + off[i]) + q, d);
-                    store_theta4(static_cast<ThetaT*>(a.theta) + off[i], q, p);
-                }
+            for (int i = 0; i < U; ++i) {
+                if (j + i * SLOTS < n) update_store<ThetaT>(a, off[i], q, p[i], sP.deviation(p[i]), dl[i], sD);
+            }
         }
     }
     if ((a.P & 3) && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) scalar_tail<ThetaT>(a, g);
 }
 
-// ---- any subgroup size (used above 256 members): two passes over the members ---------------
+// ---- subgroup means of phi alone (first half of the split-phase step) ------------------------
 //
-// Pass 1 accumulates the two sums; pass 2 re-reads phi_i together with delta_i and writes the
-// update.  The re-read hits L2 only for small subgroups; for the large ones it is used for it costs
-// 4 extra bytes of DRAM reads per parameter (28 instead of 24 bytes), and the kernel still sustains
-// a flat 5.3-5.4 TB/s of algorithmic bytes for any n, which beats clusters of 8 CTAs.
-template <typename ThetaT>
+// mean[g][p] = (1/n) sum_{j in subgroup g} phi_j[p], stored as float64.  Section 3.2 notes that
+// the slow weights of the partners are known as soon as the previous outer step has finished, so
+// this part of Eq. 2 can be exchanged early; only the pseudo-gradients have to wait for the inner
+// phase.  Read-only on phi: 4 bytes read per worker-parameter, 8/n bytes written.
+constexpr int kMeanUnroll = 4;
+
 __global__ void __launch_bounds__(kThreads)
-outer_step_any_kernel(const KArgs a) {
+group_mean_kernel(const float* __restrict__ phi, const int32_t* __restrict__ perm, int n, int64_t stride,
+                  int64_t P, double* __restrict__ mean, int64_t mean_stride, double inv_n) {
     const int g = blockIdx.y;
-    const int n = a.n;
-    const int64_t full_quads = a.P >> 2;
+    const int32_t* members = perm + (int64_t)g * n;
     const int64_t q = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    const int32_t* members = a.perm + (int64_t)g * n;
-    if (q < full_quads) {
-        float4 sD = make_float4(0.f, 0.f, 0.f, 0.f), sP = sD;
-#pragma unroll 4
-        for (int j = 0; j < n; ++j) {
-            const int64_t row = (int64_t)__ldg(members + j) * a.stride;
-            const float4 p = __ldg(reinterpret_cast<const float4*>(a.phi + row) + q);
-            const float4 t = load_theta4(static_cast<const ThetaT*>(a.theta) + row, q);
-            sD.x += p.x - t.x;  sP.x += p.x;
-            sD.y += p.y - t.y;  sP.y += p.y;
-            sD.z += p.z - t.z;  sP.z += p.z;
-            sD.w += p.w - t.w;  sP.w += p.w;
+    if (q < (P >> 2)) {
+        PairSum s;
+        s.clear();
+        for (int j = 0; j < n; j += kMeanUnroll) {
+            float4 v[kMeanUnroll];
+#pragma unroll
+            for (int i = 0; i < kMeanUnroll; ++i)
+                if (j + i < n)
+                    v[i] = __ldcs(reinterpret_cast<const float4*>(phi + (int64_t)__ldg(members + j + i) * stride) + q);
+#pragma unroll
+            for (int i = 0; i < kMeanUnroll; ++i)
+                if (j + i < n) s.add(v[i]);
         }
-        const float4 mP = make_float4(sP.x * a.inv_n, sP.y * a.inv_n, sP.z * a.inv_n, sP.w * a.inv_n);
-#pragma unroll 4
-        for (int j = 0; j < n; ++j) {
-            const int64_t row = (int64_t)__ldg(members + j) * a.stride;
-            const float4 p0 = __ldcs(reinterpret_cast<const float4*>(a.phi + row) + q);
-            const float4 d0 = __ldcs(reinterpret_cast<const float4*>(a.delta + row) + q);
-            float4 d, p;
-            p.x = update1(p0.x, d0.x, sD.x, mP.x, a, &d.x);
-            p.y = update1(p0.y, d0.y, sD.y, mP.y, a, &d.y);
-            p.z = update1(p0.z, d0.z, sD.z, mP.z, a, &d.z);
-            p.w = update1(p0.w, d0.w, sD.w, mP.w, a, &d.w);
-            __stcs(reinterpret_cast<float4*>(a.phi + row) + q, p);
-            __stcs(reinterpret_cast<float4*>(a.delta + row) + q, d);
-            store_theta4(static_cast<ThetaT*>(a.theta) + row, q, p);
+        double2* out = reinterpret_cast<double2*>(mean + (int64_t)g * mean_stride) + 2 * q;
+        out[0] = make_double2(((double)s.hi.x + (double)s.lo.x) * inv_n, ((double)s.hi.y + (double)s.lo.y) * inv_n);
+        out[1] = make_double2(((double)s.hi.z + (double)s.lo.z) * inv_n, ((double)s.hi.w + (double)s.lo.w) * inv_n);
+    }
+    if ((P & 3) && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {
+        for (int64_t c = P & ~int64_t(3); c < P; ++c) {
+            double s = 0.0;
+            for (int j = 0; j < n; ++j) s += (double)phi[(int64_t)members[j] * stride + c];
+            mean[(int64_t)g * mean_stride + c] = s * inv_n;
         }
     }
-    if ((a.P & 3) && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) scalar_tail<ThetaT>(a, g);
+}
+
+// ---- launches ---------------------------------------------------------------------------
+
+// Tiles of `quads_per_cta` quads; a trailing partial quad still needs a CTA for the scalar tail.
+bool tile_grid(const KArgs& k, int64_t quads_per_cta, int groups, dim3* grid) {
+    const int64_t quads = (k.P + 3) >> 2;
+    const int64_t tiles = (quads + quads_per_cta - 1) / quads_per_cta;
+    if (tiles > 0x7fffffffll) return false;
+    *grid = dim3((unsigned)tiles, (unsigned)groups);
+    return true;
 }
 
 template <int N, typename ThetaT, int ITEMS>
 cudaError_t launch_reg(const KArgs& k, int groups, cudaStream_t stream) {
-    const int64_t quads = (k.P + 3) >> 2;   // a trailing partial quad still needs a CTA for the tail
-    const int64_t per_cta = (int64_t)kThreads * ITEMS;
-    const int64_t tiles = (quads + per_cta - 1) / per_cta;
-    if (tiles > 0x7fffffffll) return cudaErrorInvalidConfiguration;
-    dim3 grid((unsigned)tiles, (unsigned)groups);
-    outer_step_reg_kernel<N, ThetaT, ITEMS><<<grid, kThreads, 0, stream>>>(k);
+    dim3 grid;
+    if (!tile_grid(k, (int64_t)kThreads * ITEMS, groups, &grid)) return cudaErrorInvalidConfiguration;
+    if (k.mean_phi)
+        outer_step_reg_kernel<N, ThetaT, ITEMS, true><<<grid, kThreads, 0, stream>>>(k);
+    else
+        outer_step_reg_kernel<N, ThetaT, ITEMS, false><<<grid, kThreads, 0, stream>>>(k);
     return cudaGetLastError();
 }
 
-template <int MPW, typename ThetaT, int MAXW>
-cudaError_t launch_split(const KArgs& k, int groups, int warps, int cluster, int members_per_cta,
-                         cudaStream_t stream) {
-    const int64_t quads = (k.P + 3) >> 2;
-    const int64_t tiles = (quads + 31) / 32;
-    if (tiles * cluster > 0x7fffffffll) return cudaErrorInvalidConfiguration;
-    if (cluster == 1) {
-        dim3 grid((unsigned)tiles, (unsigned)groups);
-        outer_step_split_kernel<MPW, ThetaT, false, MAXW><<<grid, warps * 32, 0, stream>>>(k, members_per_cta);
-        return cudaGetLastError();
-    }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(tiles * cluster), (unsigned)groups);
-    cfg.blockDim = dim3(warps * 32);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = cluster;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, outer_step_split_kernel<MPW, ThetaT, true, MAXW>, k, members_per_cta);
-}
-
-template <typename ThetaT, int WARPS>
-cudaError_t launch_staged(const KArgs& k, int groups, int32_t* status, cudaStream_t stream) {
-    const int64_t quads = (k.P + 3) >> 2;
-    const int64_t tiles = (quads + 31) / 32;
-    if (tiles > 0x7fffffffll) return cudaErrorInvalidConfiguration;
-    const size_t smem = (size_t)k.n * 32 * sizeof(float4);
-    cudaError_t e = cudaFuncSetAttribute(outer_step_staged_kernel<ThetaT, WARPS>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    dim3 grid((unsigned)tiles, (unsigned)groups);
-    outer_step_staged_kernel<ThetaT, WARPS><<<grid, WARPS * 32, smem, stream>>>(k, status);
+template <int MPW, typename ThetaT>
+cudaError_t launch_split(const KArgs& k, int groups, int warps, cudaStream_t stream) {
+    dim3 grid;
+    if (!tile_grid(k, 32, groups, &grid)) return cudaErrorInvalidConfiguration;
+    outer_step_split_kernel<MPW, ThetaT><<<grid, warps * 32, 0, stream>>>(k);
     return cudaGetLastError();
 }
+
+template <typename ThetaT, int WARPS, int ROWQ, int U, int MINB>
+cudaError_t launch_twopass(const KArgs& k, int groups, cudaStream_t stream) {
+    dim3 grid;
+    if (!tile_grid(k, ROWQ, groups, &grid)) return cudaErrorInvalidConfiguration;
+    outer_step_twopass_kernel<ThetaT, WARPS, ROWQ, U, MINB><<<grid, WARPS * 32, 0, stream>>>(k);
+    return cudaGetLastError();
+}
+
+constexpr int kTwoPassWideMaxN = 320;   // up to here 512-byte row segments, above 256-byte ones
 
 template <typename ThetaT>
-cudaError_t launch_any(const KArgs& k, int groups, cudaStream_t stream) {
-    const int64_t quads = (k.P + 3) >> 2;
-    const int64_t tiles = (quads + kThreads - 1) / kThreads;
-    if (tiles > 0x7fffffffll) return cudaErrorInvalidConfiguration;
-    dim3 grid((unsigned)tiles, (unsigned)groups);
-    outer_step_any_kernel<ThetaT><<<grid, kThreads, 0, stream>>>(k);
-    return cudaGetLastError();
-}
-
-template <typename ThetaT>
-cudaError_t dispatch(const KArgs& k, int groups, int32_t* status, cudaStream_t stream) {
+cudaError_t dispatch(const KArgs& k, int groups, cudaStream_t stream) {
     switch (k.n) {
-        case 1:  return launch_reg<1, ThetaT, NOLO_ITEMS_N1>(k, groups, stream);
+        case 1:  return launch_reg<1, ThetaT, 4>(k, groups, stream);
         // pairs: 2 quads per thread with fp32 theta, 1 with bf16 theta measured best (+0.7 %)
-        case 2:  return launch_reg<2, ThetaT, (sizeof(ThetaT) == 4) ? NOLO_ITEMS_N2 : 1>(k, groups, stream);
+        case 2:  return launch_reg<2, ThetaT, (sizeof(ThetaT) == 4) ? 2 : 1>(k, groups, stream);
         case 3:  return launch_reg<3, ThetaT, 1>(k, groups, stream);
-        case 4:  return launch_reg<4, ThetaT, NOLO_ITEMS_N4>(k, groups, stream);
+        case 4:  return launch_reg<4, ThetaT, 1>(k, groups, stream);
         case 5:  return launch_reg<5, ThetaT, 1>(k, groups, stream);
         case 6:  return launch_reg<6, ThetaT, 1>(k, groups, stream);
         case 7:  return launch_reg<7, ThetaT, 1>(k, groups, stream);
-        case 8:  return launch_reg<8, ThetaT, NOLO_ITEMS_N8>(k, groups, stream);
+        case 8:  return launch_reg<8, ThetaT, 1>(k, groups, stream);
         default: break;
     }
-    if (NOLO_STAGED && k.n > kSplitMembersPerCta && k.n <= NOLO_STAGED_MAX_N) {
-        if (k.n <= NOLO_STAGED_SPLIT) return launch_staged<ThetaT, 8>(k, groups, status, stream);
-        return launch_staged<ThetaT, 16>(k, groups, status, stream);
-    }
-    if (k.n <= kSplitMembersPerCta * kSplitMaxCluster) {
-        int cluster = 1;
-        while (cluster * kSplitMembersPerCta < k.n) cluster *= 2;          // 1, 2 or 4 CTAs
-        const int per_cta = (k.n + cluster - 1) / cluster;                 // members per CTA
-        const int pref = per_cta > 16 ? NOLO_SPLIT_PREF : 4;               // members per warp aimed at
-        const int G = (per_cta + pref - 1) / pref;
-        const int mpw = (per_cta + G - 1) / G;
-        constexpr int MAXW = (kSplitMembersPerCta + NOLO_SPLIT_PREF - 1) / NOLO_SPLIT_PREF;
-        static_assert(MAXW <= kSplitMaxWarps && MAXW >= 4, "CTA shape out of range");
+    if (k.n <= kSplitMaxMembers) {
+        const int pref = k.n > 16 ? kSplitPref : 4;                        // members per warp aimed at
+        const int G = (k.n + pref - 1) / pref;                             // warps
+        const int mpw = (k.n + G - 1) / G;                                 // members per warp
         switch (mpw) {
-#define NOLO_SPLIT_CASE(M) \
-    case M: return launch_split<M, ThetaT, MAXW>(k, groups, G, cluster, per_cta, stream);
-            NOLO_SPLIT_CASE(1) NOLO_SPLIT_CASE(2) NOLO_SPLIT_CASE(3) NOLO_SPLIT_CASE(4)
-            NOLO_SPLIT_CASE(5) NOLO_SPLIT_CASE(6) NOLO_SPLIT_CASE(7) NOLO_SPLIT_CASE(8)
-#undef NOLO_SPLIT_CASE
-            default: break;
+            case 1: return launch_split<1, ThetaT>(k, groups, G, stream);
+            case 2: return launch_split<2, ThetaT>(k, groups, G, stream);
+            case 3: return launch_split<3, ThetaT>(k, groups, G, stream);
+            case 4: return launch_split<4, ThetaT>(k, groups, G, stream);
+            case 5: return launch_split<5, ThetaT>(k, groups, G, stream);
+            case 6: return launch_split<6, ThetaT>(k, groups, G, stream);
+            case 7: return launch_split<7, ThetaT>(k, groups, G, stream);
+            default: return launch_split<8, ThetaT>(k, groups, G, stream);
         }
     }
-    return launch_any<ThetaT>(k, groups, stream);            // n > 256
+    if (k.n <= kTwoPassWideMaxN) return launch_twopass<ThetaT, 8, 32, 4, 3>(k, groups, stream);
+    return launch_twopass<ThetaT, 16, 16, 8, 1>(k, groups, stream);
 }
 
 }  // namespace
+
+cudaError_t launch_group_mean(const float* phi, const int32_t* perm, int W, int n, int64_t stride, int64_t P,
+                              double* mean, int64_t mean_stride, cudaStream_t stream) {
+    if (P <= 0 || W <= 0) return cudaSuccess;
+    const int64_t quads = (P + 3) >> 2;
+    const int64_t tiles = (quads + kThreads - 1) / kThreads;
+    const int groups = W / n;
+    if (tiles > 0x7fffffffll || groups > 65535) return cudaErrorInvalidConfiguration;
+    dim3 grid((unsigned)tiles, (unsigned)groups);
+    group_mean_kernel<<<grid, kThreads, 0, stream>>>(phi, perm, n, stride, P, mean, mean_stride, 1.0 / (double)n);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_outer(const OuterArgs& a, cudaStream_t stream) {
     if (a.P <= 0 || a.W <= 0) return cudaSuccess;
     KArgs k;
     k.phi = a.phi; k.theta = a.theta; k.delta = a.delta; k.perm = a.perm;
+    k.mean_phi = a.mean_phi; k.mean_stride = a.mean_stride;
     k.stride = a.stride; k.P = a.P; k.n = a.n;
     k.alpha = a.alpha; k.gamma = a.gamma;
     k.beta_over_n = a.beta / (float)a.n;
     k.inv_n = 1.0f / (float)a.n;
+    k.n_f = (float)a.n;
+    k.inv_n_d = 1.0 / (double)a.n;
     const int groups = a.W / a.n;
     if (groups > 65535) return cudaErrorInvalidConfiguration;
-    return a.theta_bf16 ? dispatch<__nv_bfloat16>(k, groups, a.status, stream)
-                        : dispatch<float>(k, groups, a.status, stream);
+    return a.theta_bf16 ? dispatch<__nv_bfloat16>(k, groups, stream) : dispatch<float>(k, groups, stream);
 }
 
 }  // namespace nolo

@@ -40,9 +40,7 @@ def main(argv=None):
                     "per-chunk normal/drift recipe (timing only; values do not affect the kernels' time)")
     args = ap.parse_args(argv)
 
-    import os
-    if not os.environ.get("NOLO_LIBRARY"):
-        build.build()
+    build.build()
     from . import binding as nolo
 
     P = args.P

@@ -128,6 +128,51 @@ def make_state(W: int, P: int, seed: int, theta_dtype=torch.float32,
     return phi, theta, delta
 
 
+MIXED_BANDS = ("near_one", "shared_base", "unit_normal", "init_scale", "zero_drift", "large_momentum")
+
+
+def make_state_mixed(W: int, P: int, seed: int, theta_dtype=torch.float32, stride: int | None = None,
+                     pad_value: float = 0.0):
+    """State whose columns cycle through six value regimes, for checking that the
+    arithmetic holds its tolerance at any ordinary weight magnitude (CPU tensors).
+
+    Column p belongs to band p % 6:
+      0 near_one        phi = 1 + N(0, 0.02^2) per worker (norm gains);
+      1 shared_base     phi = b_p + N(0, (1e-3)^2), b_p ~ U(-4, 4) common to all workers
+                        (replicas that have stayed close around weights of any size);
+      2 unit_normal     phi ~ N(0, 1) per worker (replicas far apart);
+      3 init_scale      phi ~ N(0, 0.02^2) per worker (the usual initialisation scale);
+      4 zero_drift      as band 3 but theta == phi exactly (Delta = 0; phi is made
+                        representable in theta's type);
+      5 large_momentum  as band 3 with delta ~ N(0, 1).
+    Elsewhere theta = cast(phi + N(0, (1e-3)^2)) and delta ~ N(0, (1e-4)^2).
+    Returns (phi, theta, delta) as [W, stride] tensors and the band index per column.
+    """
+    stride = padded_stride(P, 8) if stride is None else stride
+    gen = _gen("cpu", seed)
+    band = torch.arange(P) % len(MIXED_BANDS)
+    noise = lambda std: torch.empty((W, P), dtype=torch.float32).normal_(0.0, std, generator=gen)  # noqa: E731
+    base = torch.empty(P, dtype=torch.float32).uniform_(-4.0, 4.0, generator=gen)
+    cols = {
+        0: 1.0 + noise(PHI_STD),
+        1: base.unsqueeze(0) + noise(DRIFT_STD),
+        2: noise(1.0),
+    }
+    phi_v = noise(PHI_STD)
+    for b, v in cols.items():
+        phi_v = torch.where(band == b, v, phi_v)
+    zero = band == 4
+    if theta_dtype != torch.float32:
+        phi_v = torch.where(zero, phi_v.to(theta_dtype).to(torch.float32), phi_v)
+    theta_v = torch.where(zero, phi_v, phi_v + noise(DRIFT_STD)).to(theta_dtype)
+    delta_v = torch.where(band == 5, noise(1.0), noise(DELTA_STD))
+    phi = torch.full((W, stride), pad_value, dtype=torch.float32)
+    theta = torch.full((W, stride), pad_value, dtype=theta_dtype)
+    delta = torch.full((W, stride), pad_value, dtype=torch.float32)
+    phi[:, :P], theta[:, :P], delta[:, :P] = phi_v, theta_v, delta_v
+    return phi, theta, delta, band.numpy()
+
+
 def make_acts(boundaries: int, R: int, K: int, E: int, seed: int,
               dtype=torch.float32, device="cpu") -> torch.Tensor:
     """Activations at the stage boundaries, [boundaries, R, K, E], N(0, 1)."""

@@ -82,9 +82,15 @@ def test_null_handle_is_an_error_not_a_crash(lib):
 
 def test_missing_library_fails_loudly(tmp_path):
     """There is no fallback path: without the shared library the binding cannot be imported."""
+    import glob
+    import shutil
     import subprocess
     import sys
-    env = dict(os.environ, NOLO_LIBRARY=str(tmp_path / "absent.so"))
-    res = subprocess.run([sys.executable, "-c", "from paper_2506_10911_b200 import binding"], cwd=ROOT, env=env,
+    pkg = tmp_path / "paper_2506_10911_b200"          # a copy of the package without its built library
+    pkg.mkdir()
+    for f in glob.glob(os.path.join(ROOT, "paper_2506_10911_b200", "*.py")):
+        shutil.copy(f, pkg)
+    env = {k: v for k, v in os.environ.items() if k != "PYTHONPATH"}
+    res = subprocess.run([sys.executable, "-c", "from paper_2506_10911_b200 import binding"], cwd=tmp_path, env=env,
                          capture_output=True, text=True)
     assert res.returncode != 0 and "ImportError" in res.stderr and "no CPU or PyTorch fallback" in res.stderr

@@ -8,7 +8,7 @@ import torch
 
 from oracle import nolo_oracle as O
 from paper_2506_10911_b200 import synth
-from tests.helpers import assert_bf16_within_1ulp, assert_close_f32, to_np
+from tests.helpers import assert_bf16_within_1ulp, assert_close_f32, assert_outer_step_parity, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -34,7 +34,6 @@ def run_both(nolo, W, n, P, seed, step, theta_dtype=torch.float32, stride=None, 
     nolo.nolo_outer_step(h, seed, step)
     torch.cuda.synchronize()
     perm_gpu = nolo.nolo_get_groups(h)
-    assert nolo.nolo_device_status(h) == 0
     nolo.nolo_destroy(h)
 
     perm = O.draw_groups(seed, step, W, n)
@@ -43,14 +42,11 @@ def run_both(nolo, W, n, P, seed, step, theta_dtype=torch.float32, stride=None, 
     want = O.outer_step(ins[0][:, :P], ins[1][:, :P], ins[2][:, :P], perm, n, alpha, beta, gamma,
                         O.THETA_BF16 if bf16 else O.THETA_F32)
     got = [to_np(x) for x in (d_phi, d_delta, d_theta)]
-    assert_close_f32(got[0][:, :P], want[0], "phi")
-    assert_close_f32(got[1][:, :P], want[1], "delta")
+    assert_outer_step_parity(got[0][:, :P], got[1][:, :P], got[2][:, :P], want, bf16)
     if bf16:
-        assert_bf16_within_1ulp(got[2][:, :P], want[2], "theta(bf16)")
         # theta is the GPU's own phi' rounded to nearest even: exact
         assert np.array_equal(got[2][:, :P], O.f32_to_bf16_bits(got[0][:, :P]))
     else:
-        assert_close_f32(got[2][:, :P], want[2], "theta")
         assert np.array_equal(got[2][:, :P].view(np.uint32), got[0][:, :P].view(np.uint32))
     # padding columns keep their bits
     for g, i in zip((got[0], got[2], got[1]), ins):
@@ -92,10 +88,9 @@ def test_group_sizes_and_ragged_tiles(nolo, n, bf16):
 @pytest.mark.parametrize("n", [5, 6, 7, 9, 16, 17, 24, 32, 33, 48, 49, 64, 65, 96, 97, 100, 112, 113, 128, 129, 160, 192, 193, 256, 300, 512, 520])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_large_subgroups(nolo, n, bf16):
-    """8 < n <= 64 runs the kernel that splits members across warps (with masked member slots
-    when n does not fill them), 64 < n <= 192 the one that stages phi in shared memory with
-    bulk-async copies, up to 256 the thread-block-cluster kernel, above that the two-pass
-    kernel.  Two subgroups, ragged P."""
+    """8 < n <= 64 runs the kernel that shares the members out over the warps of a CTA (with
+    masked member slots when n does not fill them); above that the two-pass kernel in its two
+    shapes (up to 320 members, and beyond).  Two subgroups, ragged P."""
     dt = torch.bfloat16 if bf16 else torch.float32
     run_both(nolo, 2 * n, n, 1000 + 3, 11, 4, dt)
     if n in (16, 100, 128):
@@ -154,7 +149,7 @@ def test_nan_and_inf_propagate_within_their_subgroup_only(nolo, bf16):
 @pytest.mark.parametrize("bf16", [False, True])
 def test_guard_bands_around_every_buffer_stay_intact(nolo, W, n, bf16):
     """Each state tensor sits between two 4 KiB bands of a known pattern inside a larger
-    allocation; no kernel path (register-resident, warp-split, cluster, two-pass, ragged tail)
+    allocation; no kernel path (register-resident, warp-split, two-pass, ragged tail)
     may write outside its rows."""
     P, stride, band = 1000 + 3, 1008, 1024            # band in elements
     dt = torch.bfloat16 if bf16 else torch.float32

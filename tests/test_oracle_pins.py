@@ -142,6 +142,35 @@ def test_hand_computed_w2_p4():
         assert np.array_equal(t, p)
 
 
+def test_subgroup_mean_phi_pins():
+    """The early-exchange part of Eq. 2: the hand-computed case's mean phi, numpy's own mean
+    over the member rows, the gossip corner (alpha = beta = 0, gamma = 1 makes every member
+    equal to it), and the pull term of Eq. 2 recovered from a full step."""
+    g = read_golden("outer_step_w2_p4.txt")
+    phi = np.stack([g["phi_0"], g["phi_1"]]).astype(F32)
+    m = O.subgroup_mean_phi(phi, np.array([1, 0], dtype=np.int32), 2)
+    assert m.dtype == np.float64 and np.array_equal(m, [[2.0, 2.0, 0.0, 0.25]])   # from the golden file's header
+    phi, theta, delta = rnd_state(12, 37, 5, phi_std=1.0)
+    perm = O.draw_groups(3, 4, 12, 4)
+    m = O.subgroup_mean_phi(phi, perm, 4)
+    assert m.shape == (3, 37)
+    for gi in range(3):
+        rows = perm[gi * 4:(gi + 1) * 4]
+        np.testing.assert_allclose(m[gi], np.mean(phi[rows], axis=0, dtype=np.float64), rtol=1e-14, atol=0)
+        # a row swapped in from another group must change the mean (wrong member list is caught)
+        other = perm[((gi + 1) % 3) * 4]
+        assert not np.allclose(m[gi], np.mean(phi[[*rows[:3], other]], axis=0, dtype=np.float64))
+    p, _, _ = O.outer_step(phi, theta, delta, perm, 4, 0.0, 0.0, 1.0)
+    for gi in range(3):
+        for w in perm[gi * 4:(gi + 1) * 4]:
+            np.testing.assert_allclose(p[w], m[gi], rtol=2e-7, atol=1e-7)
+    # Eq. 2 with alpha = beta = 0: delta_i' = -gamma (phi_i - mean)  =>  mean = phi_i + delta_i'/gamma
+    _, d, _ = O.outer_step(phi, theta, delta, perm, 4, 0.0, 0.0, 0.5)
+    for gi in range(3):
+        w = perm[gi * 4]
+        np.testing.assert_allclose(phi[w].astype(np.float64) + d[w].astype(np.float64) / 0.5, m[gi], atol=3e-7)
+
+
 def test_diloco_reduction_full_group():
     """n = W: the third term of Eq. 2 vanishes only with gamma = 0 or equal
     phi; then the step is one global momentum step on the all-worker mean

@@ -56,3 +56,44 @@ def test_reference_arm_runs_on_rank0_only():
     res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
                           "--steps", "1", "--warmup", "3"], env=env, capture_output=True, text=True, timeout=120)
     assert res.returncode == 0 and res.stdout.strip() == ""
+
+
+def test_launcher_starts_every_rank_and_only_rank0_reports(tmp_path):
+    """What `bench.py --gpus N` does when it is not already under a launcher: start N rank
+    processes itself.  Two gloo ranks join, one JSON line comes back, with n_gpus 2."""
+    sys.path.insert(0, ROOT)
+    from paper_2506_10911_b200 import replicas
+    out = tmp_path / "out.txt"
+    env_before = dict(os.environ)
+    with open(out, "w") as f:
+        rc = replicas.launch(2, [sys.executable, "-m", "paper_2506_10911_b200.replicas", "--selftest", "gloo"],
+                             stdout=f, timeout=120)
+    assert rc == 0
+    assert dict(os.environ) == env_before                      # the launcher's own environment is untouched
+    lines = [ln for ln in out.read_text().splitlines() if ln.strip()]
+    assert len(lines) == 1
+    got = json.loads(lines[0])
+    assert got["n_gpus"] == 2 and got["ranks_joined"] == 2
+    assert got["ms"] == 11.0 and got["units"] == 200.0
+
+
+def test_launcher_reports_a_failing_rank(tmp_path):
+    sys.path.insert(0, ROOT)
+    from paper_2506_10911_b200 import replicas
+    code = "import os, sys, time; r = int(os.environ['RANK']); sys.exit(7) if r == 1 else time.sleep(30)"
+    assert replicas.launch(2, [sys.executable, "-c", code], timeout=60) == 7
+
+
+def test_bench_spawns_ranks_when_not_under_a_launcher(monkeypatch):
+    """bench.py --gpus 2 outside a launcher hands its own command line to replicas.launch."""
+    sys.path.insert(0, ROOT)
+    import importlib
+    bench = importlib.import_module("bench")
+    from paper_2506_10911_b200 import replicas
+    seen = {}
+    monkeypatch.setattr(replicas, "launch", lambda n, argv, **kw: seen.update(n=n, argv=argv) or 0)
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE"):
+        monkeypatch.delenv(k, raising=False)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "2", "--steps", "3"])
+    assert bench.main() == 0
+    assert seen["n"] == 2 and seen["argv"][1].endswith("bench.py") and seen["argv"][2:] == ["--gpus", "2", "--steps", "3"]

@@ -41,10 +41,16 @@ def test_static_entry_point_matches_handle_path_twice(nolo):
         want = reference_step(nolo, W, n, P, state, seed, step)
         dev = [x.clone().cuda() for x in state]
         gc.collect()                                     # leftovers of earlier tests may be freed at any time
-        before = torch.cuda.memory_allocated()
+        torch.cuda.synchronize()
+        pool_before = torch.cuda.memory_allocated()
+        free_before = torch.cuda.mem_get_info()[0]       # the driver's own count: sees any cudaMalloc
         nolo.nolo_outer_step_static(W, n, P, *HP, *dev, seed, step)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() <= before   # the call itself took nothing from torch's pool
+        assert torch.cuda.memory_allocated() <= pool_before      # nothing taken from torch's pool
+        # ... and nothing from the device behind torch's back (the driver hands memory out in
+        # blocks of 2 MiB, so even a 4-byte cudaMalloc would show; the first call's address
+        # look-up allocates nothing either)
+        assert free_before - torch.cuda.mem_get_info()[0] < (1 << 20)
         for got, w in zip(dev, want):
             # same kernels, same table: identical bits (tighter than the 2e-6 / 1e-7 parity tolerance)
             assert torch.equal(got, w)
