@@ -249,19 +249,43 @@ def sh_k(acts) -> int:
     return acts.shape[2]
 
 
+def c_oracle_step(wl, state, k: int, threads: int) -> float:
+    """The same step through the plain-C writing of the oracle (OpenMP over the columns)."""
+    from oracle import c_oracle as C
+    from oracle import nolo_oracle as O
+    W, n = wl["W"], wl["n"]
+    C.set_threads(threads)
+    t0 = time.perf_counter()
+    perm = C.draw_perm(k, k, O.DOMAIN_GROUPS, 0, 0, W)
+    phi, theta, delta, acts = state
+    C.outer_step(phi, theta, delta, perm, n, ALPHA, BETA, GAMMA, O.THETA_BF16 if wl["theta"] == "bf16" else O.THETA_F32)
+    if acts is not None:
+        C.route_forward(acts, O.draw_route(k, k, wl["stages"], W, sh_k(acts)))
+    return time.perf_counter() - t0
+
+
 def cpu_baseline(wl, sh, cols: int):
     """One oracle step on the first `cols` columns x all W rows: once on one thread, once with
-    the columns spread over all host cores."""
+    the columns spread over all host cores; then the same through the C writing of the oracle."""
     state = oracle_sample_state(wl, sh, cols)
     cores = host_cores()
     t1 = oracle_step(wl, state, 0, 1)
     tc = oracle_step(wl, state, 0, cores) if cores > 1 else t1
     W = wl["W"]
     what = "outer step + routing" if wl["M"] else "outer step"
-    return {"value": W * cols / tc, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"1 step ({what}) on {cols} of {sh['P']} columns x {W} workers, numpy float64: "
-                      f"{tc:.1f} s with the columns spread over {cores} threads, {t1:.1f} s on one thread",
-            "single_thread": {"value": W * cols / t1, "unit": UNIT, "cores": 1}}
+    rec = {"value": W * cols / tc, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"1 step ({what}) on {cols} of {sh['P']} columns x {W} workers, numpy float64: "
+                     f"{tc:.1f} s with the columns spread over {cores} threads, {t1:.1f} s on one thread",
+           "single_thread": {"value": W * cols / t1, "unit": UNIT, "cores": 1}}
+    try:
+        c1 = c_oracle_step(wl, state, 0, 1)
+        cc = min(c_oracle_step(wl, state, 0, cores) for _ in range(2))
+        rec["c_writing"] = {"value": W * cols / cc, "unit": UNIT, "cores": cores, "kind": "oracle (plain C, OpenMP)",
+                            "sample": f"the same sample: {cc:.2f} s on {cores} threads, {c1:.2f} s on one",
+                            "single_thread": {"value": W * cols / c1, "unit": UNIT, "cores": 1}}
+    except Exception as ex:    # no C compiler on the box: the numpy figures stand alone
+        rec["c_writing"] = {"value": None, "note": f"{type(ex).__name__}: {ex}"}
+    return rec
 
 
 def run_reference(args):

@@ -44,14 +44,18 @@ def build(force: bool = False, verbose: bool = False, extra: list[str] | None = 
     """Build libnolo.so if missing or older than its sources; return its path."""
     if not force and not is_stale():
         return LIB_PATH
+    tmp = f"{LIB_PATH}.{os.getpid()}.tmp"     # never leave a half-written library under the real name
     cmd = [find_nvcc(), *NVCC_FLAGS, *(extra or []),
            "-I", os.path.join(ROOT, "include"), "-I", os.path.join(HERE, "csrc"),
-           "-o", LIB_PATH, *sources()]
+           "-o", tmp, *sources()]
     if verbose:
         print(" ".join(cmd))
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
+        if os.path.exists(tmp):
+            os.unlink(tmp)
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+    os.replace(tmp, LIB_PATH)
     if verbose:
         print(res.stdout + res.stderr)
     return LIB_PATH

@@ -12,15 +12,9 @@ namespace nolo {
 
 namespace {
 
-#ifndef NOLO_DIV_ITEMS
-#define NOLO_DIV_ITEMS 4
-#endif
-#ifndef NOLO_DIV_UNROLL
-#define NOLO_DIV_UNROLL 4
-#endif
 constexpr int kThreads = 256;
-constexpr int kItems = NOLO_DIV_ITEMS;       // quads per thread
-constexpr int kUnroll = NOLO_DIV_UNROLL;    // worker rows in flight per thread
+constexpr int kItems = 4;     // quads per thread
+constexpr int kUnroll = 4;    // worker rows in flight per thread
 
 struct Welford4 {
     float4 mean, m2;

@@ -10,11 +10,8 @@ namespace nolo {
 
 namespace {
 
-#ifndef NOLO_ROUTE_ILP
-#define NOLO_ROUTE_ILP 4
-#endif
 constexpr int kThreads = 256;
-constexpr int kVecPerThread = NOLO_ROUTE_ILP;
+constexpr int kVecPerThread = 4;                      // 128-bit loads in flight per thread
 constexpr int kTileVecs = kThreads * kVecPerThread;   // vectors per tile
 
 struct Blocks {

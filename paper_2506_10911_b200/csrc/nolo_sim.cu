@@ -16,10 +16,7 @@ namespace nolo {
 
 namespace {
 
-#ifndef NOLO_TREE_THREADS
-#define NOLO_TREE_THREADS 128
-#endif
-constexpr int kTreeThreads = NOLO_TREE_THREADS;   // small CTAs: the upper tree levels leave few threads busy
+constexpr int kTreeThreads = 128;   // small CTAs: the upper tree levels leave few threads busy
 constexpr uint64_t kDomainTree = 3;
 constexpr uint64_t kDomainStraggler = 4;
 
