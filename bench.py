@@ -83,9 +83,9 @@ def kernel_name(n: int, theta: str) -> str:
         return f"outer_step_reg_kernel<{n},{t},{items}>"
     if n <= 64:
         return f"outer_step_split_kernel<{t}> (warps share the subgroup)"
-    if n <= 320:
-        return f"outer_step_twopass_kernel<{t},8 warps,32 quads,4 rows> (second read of phi from L1/L2)"
-    return f"outer_step_twopass_kernel<{t},16 warps,16 quads,8 rows> (second read of phi from L1/L2)"
+    shape = ("8 warps,32 quads,4 rows" if n <= 128 else "8 warps,32 quads,8 rows" if n <= 224 else
+             "8 warps,16 quads,8 rows" if n <= 640 else "16 warps,16 quads,8 rows")
+    return f"outer_step_twopass_kernel<{t},{shape}> (second read of phi from L1/L2)"
 
 
 def workload_shape(wl):

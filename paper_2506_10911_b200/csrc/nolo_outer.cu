@@ -361,12 +361,26 @@ outer_step_split_kernel(const KArgs a) {
 // slot s walks members s, s + SLOTS, ... in chunks of U rows in flight.  Pass 1 reads phi and
 // theta and accumulates the two sums; the slots' partial sums meet in shared memory; pass 2
 // reads phi again together with delta and writes the update.  Between the two reads of a phi
-// element lie only the other rows of the same CTA's tile (n x ROWQ x 16 bytes, 32-128 KB for the
-// shapes used), so the second read is served by L1 or L2: profiled DRAM traffic equals the
-// algorithmic 24 / 20 bytes per worker-parameter, and nothing has to be parked in registers or
-// shared memory, whatever n is.  No bulk copies, no clusters and no waits other than the one CTA
-// barrier.  Shapes (by measurement): 8 warps x 32 quads x 4 rows in flight, 3 CTAs per SM, up to
-// 320 members; 16 warps x 16 quads x 8 rows above (narrower segments keep the tile cacheable).
+// element lie only the other rows of the same CTA's tile (n x ROWQ x 16 bytes), so the second
+// read is served by L1 or L2 as long as the tiles of all resident CTAs fit there: profiled DRAM
+// traffic equals the algorithmic 24 / 20 bytes per worker-parameter, and nothing has to be parked
+// in registers or shared memory, whatever n is.  The first chunk of pass 2 depends on no sum, so
+// its loads are issued before the partial sums meet and are in flight across the CTA barrier.
+// No bulk copies, no clusters and no waits other than that one barrier.
+//
+// The shape trades three things: bytes in flight (warps x U), the width of a row segment (DRAM
+// likes 512 bytes better than 256) and the L2 footprint of the resident tiles
+// (CTAs per SM x n x ROWQ x 16 bytes x 148 SMs), which must stay well below the 126 MB of L2 or
+// the re-read goes to DRAM.  Measured best on B200 (fraction of a plain copy, float32 / bfloat16
+// theta): 8 warps x 32 quads x 4 rows, 3 CTAs per SM up to 128 members (0.94); 8 rows in flight
+// and 2 CTAs per SM up to 224 (0.92 - 0.90); 16-quad segments up to 640 (0.93 - 0.88); above that
+// 16 warps x 16 quads x 8 rows, one CTA per SM (0.92 - 0.84 at 1024).  Tried and measured slower on
+// this access pattern: rings of asynchronous copies (cp.async) that keep several chunks in
+// flight per thread (same rate: the kernel is not short of loads in flight), phi parked in shared
+// memory, and phi parked in tensor memory (tcgen05.st / tcgen05.ld; exact, but two CTAs of eight
+// warps per SM are too few warps: 0.78 - 0.85).  Even with the re-read of phi left out altogether
+// the same loops reach only 0.92 / 0.91 / 0.89 of a plain copy at n = 128 / 256 / 1024: what is lost is
+// lost to streaming n x 3 rows in 512-byte pieces, not to the second read.
 template <typename ThetaT, int WARPS, int ROWQ, int U, int MINB>
 __global__ void __launch_bounds__(WARPS * 32, MINB)
 outer_step_twopass_kernel(const KArgs a) {
@@ -409,6 +423,21 @@ outer_step_twopass_kernel(const KArgs a) {
             }
         }
     }
+    // pass 2, chunk by chunk: phi (from L1 / L2) and delta of U rows
+    float4 p2[U], d2[U];
+    int64_t off2[U];
+    auto load_chunk = [&](int j) {
+#pragma unroll
+        for (int i = 0; i < U; ++i) {
+            const int jj = j + i * SLOTS;
+            if (jj < n) {
+                off2[i] = (int64_t)__ldg(members + jj) * a.stride;
+                p2[i] = __ldcs(reinterpret_cast<const float4*>(a.phi + off2[i]) + q);
+                d2[i] = __ldcs(reinterpret_cast<const float4*>(a.delta + off2[i]) + q);
+            }
+        }
+    };
+    if (ok) load_chunk(slot);      // in flight while the partial sums meet
     // the slots of one warp that share a quad (fixed order), then the warps through shared memory
 #pragma unroll
     for (int o = ROWQ; o < 32; o <<= 1) {
@@ -448,20 +477,10 @@ outer_step_twopass_kernel(const KArgs a) {
         if (a.mean_phi) sP = load_prepared_mean(a, g, q);
         else sP.divide(a);
         for (int j = slot; j < n; j += SLOTS * U) {
-            float4 p[U], dl[U];
-            int64_t off[U];
+            if (j != slot) load_chunk(j);
 #pragma unroll
             for (int i = 0; i < U; ++i) {
-                const int jj = j + i * SLOTS;
-                if (jj < n) {
-                    off[i] = (int64_t)__ldg(members + jj) * a.stride;
-                    p[i] = __ldcs(reinterpret_cast<const float4*>(a.phi + off[i]) + q);
-                    dl[i] = __ldcs(reinterpret_cast<const float4*>(a.delta + off[i]) + q);
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < U; ++i) {
-                if (j + i * SLOTS < n) update_store<ThetaT>(a, off[i], q, p[i], sP.deviation(p[i]), dl[i], sD);
+                if (j + i * SLOTS < n) update_store<ThetaT>(a, off2[i], q, p2[i], sP.deviation(p2[i]), d2[i], sD);
             }
         }
     }
@@ -546,7 +565,10 @@ cudaError_t launch_twopass(const KArgs& k, int groups, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
-constexpr int kTwoPassWideMaxN = 320;   // up to here 512-byte row segments, above 256-byte ones
+// Subgroup sizes up to which each two-pass shape is used (by measurement, see the kernel's comment).
+constexpr int kTwoPassMaxN4Rows = 128;   // 8 warps x 32 quads x 4 rows in flight, 3 CTAs per SM
+constexpr int kTwoPassMaxN32Quads = 224; // 8 warps x 32 quads x 8 rows, 2 CTAs per SM
+constexpr int kTwoPassMaxN8Warps = 640;  // 8 warps x 16 quads x 8 rows, 2 CTAs per SM; above: 16 warps, 1 CTA per SM
 
 template <typename ThetaT>
 cudaError_t dispatch(const KArgs& k, int groups, cudaStream_t stream) {
@@ -577,7 +599,9 @@ cudaError_t dispatch(const KArgs& k, int groups, cudaStream_t stream) {
             default: return launch_split<8, ThetaT>(k, groups, G, stream);
         }
     }
-    if (k.n <= kTwoPassWideMaxN) return launch_twopass<ThetaT, 8, 32, 4, 3>(k, groups, stream);
+    if (k.n <= kTwoPassMaxN4Rows) return launch_twopass<ThetaT, 8, 32, 4, 3>(k, groups, stream);
+    if (k.n <= kTwoPassMaxN32Quads) return launch_twopass<ThetaT, 8, 32, 8, 2>(k, groups, stream);
+    if (k.n <= kTwoPassMaxN8Warps) return launch_twopass<ThetaT, 8, 16, 8, 2>(k, groups, stream);
     return launch_twopass<ThetaT, 16, 16, 8, 1>(k, groups, stream);
 }
 

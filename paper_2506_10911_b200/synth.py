@@ -51,9 +51,15 @@ def stage_params(name: str, stages: int) -> int:
 
 
 def padded_stride(P: int, multiple: int = 64) -> int:
-    """Row stride in elements: P rounded up so that every row starts on a
-    256-byte boundary for 4-byte elements."""
-    return (P + multiple - 1) // multiple * multiple
+    """Row stride in elements: P rounded up to a multiple of ``multiple`` (64 elements: every
+    row starts on a 256-byte boundary).  A stride that comes out as a multiple of 2^17 elements
+    (512 KiB rows or a multiple) gets 1024 more: rows that far apart by an exact power of two map
+    the same column of every row to the same memory channels, which measured 4-8 % slower when
+    hundreds of rows are streamed side by side; any smaller offset between rows removes it."""
+    stride = (P + multiple - 1) // multiple * multiple
+    if multiple >= 64 and stride % (1 << 17) == 0:
+        stride += 1024
+    return stride
 
 
 def _gen(device, seed: int) -> torch.Generator:

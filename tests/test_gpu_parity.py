@@ -85,12 +85,13 @@ def test_group_sizes_and_ragged_tiles(nolo, n, bf16):
     run_both(nolo, W, n, 5 * 1024 + 3, 7, 3, dt, stride=5 * 1024 + 16)
 
 
-@pytest.mark.parametrize("n", [5, 6, 7, 9, 16, 17, 24, 32, 33, 48, 49, 64, 65, 96, 97, 100, 112, 113, 128, 129, 160, 192, 193, 256, 300, 512, 520])
+@pytest.mark.parametrize("n", [5, 6, 7, 9, 16, 17, 24, 32, 33, 48, 49, 64, 65, 96, 97, 100, 112, 113, 128, 129, 160, 192, 193, 224, 225, 256, 300,
+                               512, 520, 640, 641])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_large_subgroups(nolo, n, bf16):
     """8 < n <= 64 runs the kernel that shares the members out over the warps of a CTA (with
-    masked member slots when n does not fill them); above that the two-pass kernel in its two
-    shapes (up to 320 members, and beyond).  Two subgroups, ragged P."""
+    masked member slots when n does not fill them); above that the two-pass kernel in its four
+    shapes (up to 128, 224 and 640 members, and beyond).  Two subgroups, ragged P."""
     dt = torch.bfloat16 if bf16 else torch.float32
     run_both(nolo, 2 * n, n, 1000 + 3, 11, 4, dt)
     if n in (16, 100, 128):
