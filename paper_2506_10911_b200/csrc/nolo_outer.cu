@@ -493,36 +493,69 @@ outer_step_twopass_kernel(const KArgs a) {
 // the slow weights of the partners are known as soon as the previous outer step has finished, so
 // this part of Eq. 2 can be exchanged early; only the pseudo-gradients have to wait for the inner
 // phase.  Read-only on phi: 4 bytes read per worker-parameter, 8/n bytes written.
-constexpr int kMeanUnroll = 4;
+constexpr int kMeanUnroll = 4;   // member rows in flight per quad
 
+// Four consecutive float64 means with one 256-bit store (one whole 32-byte sector per lane) where
+// the row is 32-byte aligned, else as two 128-bit stores.
+template <bool WIDE>
+__device__ __forceinline__ void store_mean4(double* out, double a, double b, double c, double d) {
+    if (WIDE) {
+        asm volatile("st.global.cs.v4.f64 [%0], {%1, %2, %3, %4};" :: "l"(out), "d"(a), "d"(b), "d"(c), "d"(d) : "memory");
+    } else {
+        __stcs(reinterpret_cast<double2*>(out), make_double2(a, b));
+        __stcs(reinterpret_cast<double2*>(out) + 1, make_double2(c, d));
+    }
+}
+
+// ITEMS quads per thread, 256 quads apart: small subgroups have few rows to keep in flight per
+// quad, so each thread takes two quads up to n = 4.
+template <int ITEMS, bool WIDE>
 __global__ void __launch_bounds__(kThreads)
 group_mean_kernel(const float* __restrict__ phi, const int32_t* __restrict__ perm, int n, int64_t stride,
                   int64_t P, double* __restrict__ mean, int64_t mean_stride, double inv_n) {
     const int g = blockIdx.y;
     const int32_t* members = perm + (int64_t)g * n;
-    const int64_t q = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (q < (P >> 2)) {
-        PairSum s;
-        s.clear();
-        for (int j = 0; j < n; j += kMeanUnroll) {
-            float4 v[kMeanUnroll];
+    const int64_t q0 = (int64_t)blockIdx.x * (kThreads * ITEMS) + threadIdx.x;
+    const int64_t quads = P >> 2;
+    PairSum s[ITEMS];
 #pragma unroll
-            for (int i = 0; i < kMeanUnroll; ++i)
-                if (j + i < n)
-                    v[i] = __ldcs(reinterpret_cast<const float4*>(phi + (int64_t)__ldg(members + j + i) * stride) + q);
+    for (int it = 0; it < ITEMS; ++it) s[it].clear();
+    for (int j = 0; j < n; j += kMeanUnroll) {
+        float4 v[ITEMS][kMeanUnroll];
 #pragma unroll
-            for (int i = 0; i < kMeanUnroll; ++i)
-                if (j + i < n) s.add(v[i]);
+        for (int i = 0; i < kMeanUnroll; ++i) {
+            if (j + i < n) {
+                const float4* row = reinterpret_cast<const float4*>(phi + (int64_t)__ldg(members + j + i) * stride);
+#pragma unroll
+                for (int it = 0; it < ITEMS; ++it) {
+                    const int64_t q = q0 + (int64_t)it * kThreads;
+                    if (q < quads) v[it][i] = __ldcs(row + q);
+                }
+            }
         }
-        double2* out = reinterpret_cast<double2*>(mean + (int64_t)g * mean_stride) + 2 * q;
-        out[0] = make_double2(((double)s.hi.x + (double)s.lo.x) * inv_n, ((double)s.hi.y + (double)s.lo.y) * inv_n);
-        out[1] = make_double2(((double)s.hi.z + (double)s.lo.z) * inv_n, ((double)s.hi.w + (double)s.lo.w) * inv_n);
+#pragma unroll
+        for (int i = 0; i < kMeanUnroll; ++i) {
+            if (j + i < n) {
+#pragma unroll
+                for (int it = 0; it < ITEMS; ++it)
+                    if (q0 + (int64_t)it * kThreads < quads) s[it].add(v[it][i]);
+            }
+        }
+    }
+#pragma unroll
+    for (int it = 0; it < ITEMS; ++it) {
+        const int64_t q = q0 + (int64_t)it * kThreads;
+        if (q < quads) {
+            store_mean4<WIDE>(mean + (int64_t)g * mean_stride + 4 * q,
+                              ((double)s[it].hi.x + (double)s[it].lo.x) * inv_n, ((double)s[it].hi.y + (double)s[it].lo.y) * inv_n,
+                              ((double)s[it].hi.z + (double)s[it].lo.z) * inv_n, ((double)s[it].hi.w + (double)s[it].lo.w) * inv_n);
+        }
     }
     if ((P & 3) && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {
         for (int64_t c = P & ~int64_t(3); c < P; ++c) {
-            double s = 0.0;
-            for (int j = 0; j < n; ++j) s += (double)phi[(int64_t)members[j] * stride + c];
-            mean[(int64_t)g * mean_stride + c] = s * inv_n;
+            double t = 0.0;
+            for (int j = 0; j < n; ++j) t += (double)phi[(int64_t)members[j] * stride + c];
+            mean[(int64_t)g * mean_stride + c] = t * inv_n;
         }
     }
 }
@@ -610,12 +643,20 @@ cudaError_t dispatch(const KArgs& k, int groups, cudaStream_t stream) {
 cudaError_t launch_group_mean(const float* phi, const int32_t* perm, int W, int n, int64_t stride, int64_t P,
                               double* mean, int64_t mean_stride, cudaStream_t stream) {
     if (P <= 0 || W <= 0) return cudaSuccess;
+    const int items = n <= 4 ? 2 : 1;
     const int64_t quads = (P + 3) >> 2;
-    const int64_t tiles = (quads + kThreads - 1) / kThreads;
+    const int64_t per_cta = (int64_t)kThreads * items;
+    const int64_t tiles = (quads + per_cta - 1) / per_cta;
     const int groups = W / n;
     if (tiles > 0x7fffffffll || groups > 65535) return cudaErrorInvalidConfiguration;
     dim3 grid((unsigned)tiles, (unsigned)groups);
-    group_mean_kernel<<<grid, kThreads, 0, stream>>>(phi, perm, n, stride, P, mean, mean_stride, 1.0 / (double)n);
+    const double inv_n = 1.0 / (double)n;
+    // rows of the means are 32-byte aligned when the base is (the stride is a multiple of 64 bytes)
+    const bool wide = (reinterpret_cast<uintptr_t>(mean) & 31u) == 0;
+#define NOLO_MEAN_LAUNCH(I, WD) group_mean_kernel<I, WD><<<grid, kThreads, 0, stream>>>(phi, perm, n, stride, P, mean, mean_stride, inv_n)
+    if (items == 2) { if (wide) NOLO_MEAN_LAUNCH(2, true); else NOLO_MEAN_LAUNCH(2, false); }
+    else { if (wide) NOLO_MEAN_LAUNCH(1, true); else NOLO_MEAN_LAUNCH(1, false); }
+#undef NOLO_MEAN_LAUNCH
     return cudaGetLastError();
 }
 

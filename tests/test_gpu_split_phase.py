@@ -70,6 +70,29 @@ def test_prepared_and_fused_steps_agree_over_consecutive_steps(nolo):
     nolo.nolo_destroy(hs)
 
 
+@pytest.mark.parametrize("n", [2, 8])
+def test_means_buffer_aligned_to_16_bytes_only(nolo, n):
+    """The means are stored 32 bytes at a time when their rows allow it; a buffer that starts on
+    a 16-byte boundary only takes the other store path and must give the same means."""
+    W, P = 2 * n, 2051
+    phi, theta, delta = synth.make_state(W, P, 77)
+    dev = [x.cuda() for x in (phi, theta, delta)]
+    stride = synth.padded_stride(P, 8)
+    backing = torch.full((2 + (W // n) * stride,), float("nan"), dtype=torch.float64, device="cuda")
+    mean = backing[2:].view(W // n, stride)
+    assert mean.data_ptr() % 32 == 16
+    h = nolo.nolo_create(W, n, P, 1, *HP)
+    nolo.nolo_bind_state(h, *dev)
+    nolo.nolo_bind_prepared(h, mean)
+    nolo.nolo_outer_prepare(h, 3, 3)
+    torch.cuda.synchronize()
+    got = mean.cpu().numpy()
+    want = O.subgroup_mean_phi(to_np(phi)[:, :P], O.draw_groups(3, 3, W, n), n)
+    np.testing.assert_allclose(got[:, :P], want, rtol=1e-12, atol=1e-14)
+    assert np.isnan(got[:, P:]).all() and np.isnan(backing[:2].cpu().numpy()).all()     # nothing else written
+    nolo.nolo_destroy(h)
+
+
 def test_prepared_means_are_refused_when_stale_or_mismatched(nolo):
     W, n, P = 8, 4, 1000
     dev = [x.cuda() for x in synth.make_state(W, P, 2)]
