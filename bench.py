@@ -66,8 +66,8 @@ WORKLOADS = [
 # the captured launch); traffic grows in proportion to the columns processed.  None = not captured
 # since the kernel last changed.
 PROFILED_DRAM_BYTES_PER_PARAM = {
-    "outer_step_reg_kernel<2,bf16,1>": None,
-    "outer_step_reg_kernel<4,float,1>": None,
+    "outer_step_reg_kernel<2,bf16,1>": 2.627498e9 / (16 * 8388608),     # 19.58
+    "outer_step_reg_kernel<4,float,1>": 1.553978e9 / (8 * 8388608),      # 23.16
 }
 
 
@@ -611,7 +611,11 @@ def run_ours(args):
     torch.cuda.empty_cache()
     if world == 1 and not args.no_configs:
         args.headline = wl["name"]
-        line["configs"] = extra_configs(nolo, dev, peak, copy_gbs, args)
+        headline_rec = stats_record(f"{wl['name']} (the headline workload above): W={W} n={n} {wl['text']}", kname,
+                                    outer_stats, outer_cnt, bpp * W * P, peak, copy_gbs, W=W, n=n, P=P,
+                                    theta=wl["theta"], resident_gb=sh["state_bytes"] / GB,
+                                    params_per_s=W * P / (per_launch_ms * 1e-3))
+        line["configs"] = [headline_rec] + extra_configs(nolo, dev, peak, copy_gbs, args)
     if args.no_cpu_baseline or world > 1:
         line["cpu_baseline"] = None
     else:

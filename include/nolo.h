@@ -107,8 +107,10 @@ int nolo_bind_state(nolo_handle* h, void* phi, void* theta, void* delta,
  * float32 arithmetic, with the subgroup mean of phi carried to about 46 bits so
  * that gamma (phi_i - mean) is accurate for weights of any magnitude; sums in a
  * fixed order (results are reproducible bit for bit); every element of every
- * worker is fetched from device memory once and written once.  Asynchronous.  Errors: NOLO_EINVAL (NULL handle), NOLO_ESTATE (no
- * state bound), NOLO_ECUDA (launch failure).
+ * worker is fetched from device memory once and written once (subgroups of
+ * more than 64 members request phi a second time, which the caches serve).
+ * Asynchronous.  Errors: NOLO_EINVAL (NULL handle), NOLO_ESTATE (no state
+ * bound), NOLO_ECUDA (launch failure).
  */
 int nolo_outer_step(nolo_handle* h, uint64_t seed, uint64_t step);
 
@@ -340,8 +342,8 @@ int nolo_sim_straggler(int W, int n, int H, int T, double mu, double sigma, int6
 
 /*
  * (Measurement aid; the paper has no counterpart.)  Times a plain
- * device-to-device copy of `bytes` bytes with the routing kernel's access
- * pattern (one-shot grid, 128-bit streaming loads and stores): 3 warm-up
+ * device-to-device copy of `bytes` bytes (a one-shot grid of 128-bit streaming
+ * loads and stores, two per thread: the fastest plain copy found): 3 warm-up
  * copies, then `iters` copies between CUDA events on `stream`.  The bandwidth
  * 2 * bytes / time is the practical HBM ceiling for a half-read, half-write
  * kernel on this device, against which the other kernels can be read.

@@ -60,7 +60,7 @@ struct RouteArgs {
 
 cudaError_t launch_route(const RouteArgs& a, cudaStream_t stream);
 
-// Plain copy of `bytes` (a multiple of 16) with the routing kernel's access pattern.
+// Plain copy of `bytes` (a multiple of 16): one-shot grid, 128-bit streaming loads and stores.
 cudaError_t launch_copy_probe(const void* in, void* out, int64_t bytes, cudaStream_t stream);
 
 // Replica divergence of phi (Fig. 3b): out2[0] = mean over parameters of the across-worker
