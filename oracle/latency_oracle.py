@@ -20,14 +20,18 @@ Two simulations, as the paper describes them:
   steps; NoLoCo only waits for the members of its random subgroup of n.
   Returns the time for all workers to finish T outer iterations under each.
 
-Random numbers (the paper gives none): uniform u = ((x >> 11) + 0.5) 2^-53
-from 64-bit Philox words, normal z = sqrt(-2 ln u1) cos(2 pi u2) (Box-Muller)
-from words 0 and 1 of one Philox block, t = exp(mu + sigma z).
-  tree:       counter (node, trial, phase, 3), key (seed, 0); node = heap index
-              of the child end of the edge (2 .. 2W-1), phase 0 up / 1 down
-  straggler:  counter (inner step k, worker w, outer step t, 4), key (seed, trial);
-              subgroups of outer step t: the library's permutation draw with
-              (seed, step = t, boundary = trial).
+Random numbers (the paper gives none; the library defines them).  One Philox
+block of four 64-bit words gives four log-normal times: uniform
+u = ((x >> 11) + 0.5) 2^-53 from each word; Box-Muller on the word pairs (0, 1)
+and (2, 3): r = sqrt(-2 ln u_a), z = r cos(2 pi u_b) and r sin(2 pi u_b), so the
+block's four normals are [r01 cos, r01 sin, r23 cos, r23 sin]; t = exp(mu + sigma z).
+Sample number j of a stream lives in block j // 4, position j % 4.
+  tree:       stream index = heap index of the child end of the edge
+              (2 .. 2W-1); counter (node // 4, trial, phase, 3), key (seed, 0);
+              phase 0 up / 1 down
+  straggler:  stream index = inner step k; counter (k // 4, worker w, outer step t, 4),
+              key (seed, trial); subgroups of outer step t: the library's
+              permutation draw with (seed, step = t, boundary = trial).
 """
 
 from __future__ import annotations
@@ -78,9 +82,26 @@ def uniform_open(x):
     return ((np.asarray(x, dtype=np.uint64) >> np.uint64(11)).astype(np.float64) + 0.5) * 2.0 ** -53
 
 
-def lognormal_from_words(w0, w1, mu, sigma):
-    z = np.sqrt(-2.0 * np.log(uniform_open(w0))) * np.cos(2.0 * np.pi * uniform_open(w1))
-    return np.exp(mu + sigma * z)
+def lognormal4_from_block(w0, w1, w2, w3, mu, sigma):
+    """The four log-normal times of one Philox block (arrays broadcast): stacked on a new last
+    axis in the order [cos of pair (0,1), sin of pair (0,1), cos of pair (2,3), sin of pair (2,3)]."""
+    z = []
+    for a, b in ((w0, w1), (w2, w3)):
+        r = np.sqrt(-2.0 * np.log(uniform_open(a)))
+        ang = 2.0 * np.pi * uniform_open(b)
+        z += [r * np.cos(ang), r * np.sin(ang)]
+    return np.exp(mu + sigma * np.stack(z, axis=-1))
+
+
+def stream_times(count, c1, c2, domain, mu, sigma, k0, k1):
+    """Samples 0 .. count-1 of the stream with counter words (block, c1, c2, domain) and key
+    (k0, k1); c1 may be an array (one stream per entry, result [len(c1), count])."""
+    blocks = np.arange((count + 3) // 4, dtype=np.uint64)
+    c1 = np.asarray(c1, dtype=np.uint64)
+    w = philox4x64_10_np(blocks if c1.ndim == 0 else blocks[None, :], c1 if c1.ndim == 0 else c1[:, None],
+                         c2, domain, k0, k1)
+    t = lognormal4_from_block(*w, mu, sigma)                  # [..., blocks, 4]
+    return t.reshape(t.shape[:-2] + (-1,))[..., :count]
 
 
 def expected_pair_exchange(mu, sigma):
@@ -92,9 +113,7 @@ def expected_pair_exchange(mu, sigma):
 
 def message_times(W, trial, phase, mu, sigma, seed):
     """Times of the 2W-2 messages of one phase of one trial, indexed by child node (2..2W-1)."""
-    node = np.arange(2 * W, dtype=np.uint64)
-    w0, w1, _, _ = philox4x64_10_np(node, trial, phase, DOMAIN_TREE, seed, 0)
-    return lognormal_from_words(w0, w1, mu, sigma)
+    return stream_times(2 * W, trial, phase, DOMAIN_TREE, mu, sigma, seed, 0)
 
 
 def sim_tree_allreduce(W, mu, sigma, trials, seed):
@@ -120,14 +139,12 @@ def sim_straggler(W, n, H, T, mu, sigma, trials, seed):
     """[trials, 2]: time for all workers to finish T outer iterations of H inner
     steps under (global barrier every outer step, wait only for the subgroup)."""
     out = np.empty((trials, 2), dtype=np.float64)
-    k = np.arange(H, dtype=np.uint64)[None, :]
-    w = np.arange(W, dtype=np.uint64)[:, None]
+    w = np.arange(W, dtype=np.uint64)
     for s in range(trials):
         barrier_clock = 0.0
         clock = np.zeros(W)
         for t in range(T):
-            w0, w1, _, _ = philox4x64_10_np(k, w, t, DOMAIN_STRAGGLER, seed, s)
-            steps = lognormal_from_words(w0, w1, mu, sigma)      # [W, H]
+            steps = stream_times(H, w, t, DOMAIN_STRAGGLER, mu, sigma, seed, s)      # [W, H]
             work = np.zeros(W)
             for kk in range(H):                                   # same summation order as a loop
                 work = work + steps[:, kk]
