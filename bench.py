@@ -423,6 +423,55 @@ def extra_configs(nolo, dev, peak, copy_gbs, args):
     return out
 
 
+# Issue-slot bound of the simulation kernels.  Thread-instructions per log-normal sample, from a
+# profiler capture of each kernel (warp instructions x 32 / samples): the straggler kernel spends a
+# quarter of a Philox block (ten rounds of two 64 x 64 -> 128-bit products) and half a logarithm,
+# square root and sine/cosine pair plus one exponential in float64 per sample; the tree kernel
+# computes every block twice (one thread per sibling pair) and walks the tree.  The bound is
+# SMs x 4 schedulers x 32 lanes x SM clock / that count.
+SIM_THREAD_INSTR_PER_SAMPLE = {"straggler_kernel": 278.0, "tree_allreduce_kernel": 420.0}
+
+
+def sim_records(nolo):
+    """The paper's two latency simulations at Fig. 5's largest size: device time between CUDA
+    events around the (synchronous) calls, log-normal samples per second, and the fraction of the
+    issue-slot bound."""
+    import math
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            sm_hz = float(json.load(f)["sm_max_mhz"]) * 1e6
+    except Exception:
+        sm_hz = 1.965e9
+    sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    slots = sms * 4 * 32 * sm_hz                                  # thread-instructions per second
+    out = []
+    cases = [("simulation: straggler barrier (Fig. 5b), W=1024 n=2 H=100 T=250, 592 trials", "straggler_kernel",
+              lambda: nolo.nolo_sim_straggler(1024, 2, 100, 250, 1.0, math.sqrt(0.5), 592, 0), 592 * 1024 * 100 * 250),
+             ("simulation: tree all-reduce vs pair exchange (Fig. 5a), W=1024 sigma=1, 100000 trials",
+              "tree_allreduce_kernel", lambda: nolo.nolo_sim_tree_allreduce(1024, 0.0, 1.0, 100_000, 0),
+              100_000 * (4 * 1024 - 4))]
+    for name, kernel, call, samples in cases:
+        call()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        res = call()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        rate = samples / (ms * 1e-3)
+        peak = slots / SIM_THREAD_INSTR_PER_SAMPLE[kernel]
+        rec = {"name": name, "kernel": kernel, "ms": ms, "samples": samples, "samples_per_s": rate,
+               "roofline": {"bound": "alu", "achieved": rate / 1e9, "peak": peak / 1e9, "unit": "G samples/s",
+                            "frac": rate / peak, "peak_kind": "issue slots: SMs x 4 schedulers x 32 lanes x SM clock / "
+                                                              f"{SIM_THREAD_INSTR_PER_SAMPLE[kernel]:.0f} profiled thread-instructions per sample"}}
+        if kernel == "straggler_kernel":
+            rec["barrier_over_subgroup"] = res[0] / res[1]
+        else:
+            rec["tree_over_pair"] = res[0] / nolo.nolo_expected_pair_exchange(0.0, 1.0)
+        out.append(rec)
+    return out
+
+
 def measure_e2e(nolo, args, wl, sh, state, acts, acts_out, world, dev):
     """End to end: state and activations in pinned host memory, through the host entry points.
     The full state (>100 GB) cannot be page-locked on the host, so a column slice of it is
@@ -616,6 +665,7 @@ def run_ours(args):
                                     theta=wl["theta"], resident_gb=sh["state_bytes"] / GB,
                                     params_per_s=W * P / (per_launch_ms * 1e-3))
         line["configs"] = [headline_rec] + extra_configs(nolo, dev, peak, copy_gbs, args)
+        line["simulations"] = sim_records(nolo)
     if args.no_cpu_baseline or world > 1:
         line["cpu_baseline"] = None
     else:

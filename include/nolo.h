@@ -296,10 +296,13 @@ int nolo_divergence(nolo_handle* h, double* host_out);
  * With constant message time t_c this is the paper's 2 t_c log2(W); with W = 2
  * it is the pair exchange of local averaging, max(t1,t2) + max(t3,t4).
  *   W       power of two, 2..NOLO_MAX_WORKERS;  sigma >= 0;  trials 1..2^24
- *   seed    random stream: the message on the edge above heap node c (2..2W-1)
- *           in phase p (0 up, 1 down) of trial s uses philox4x64-10(counter =
- *           (c, s, p, 3), key = (seed, 0)); u = ((word >> 11) + 0.5) 2^-53;
- *           z = sqrt(-2 ln u(word0)) cos(2 pi u(word1)); t = exp(mu + sigma z)
+ *   seed    random stream.  One philox4x64-10 block gives four times: each
+ *           word x gives u = ((x >> 11) + 0.5) 2^-53; Box-Muller on the word
+ *           pairs (0,1) and (2,3), r = sqrt(-2 ln u_a), gives the normals
+ *           z = [r01 cos, r01 sin, r23 cos, r23 sin] of the angle 2 pi u_b;
+ *           t = exp(mu + sigma z).  The message on the edge above heap node c
+ *           (2..2W-1) in phase p (0 up, 1 down) of trial s is position c % 4 of
+ *           the block with counter (c / 4, s, p, 3) and key (seed, 0)
  *   stream  cudaStream_t for the kernels
  *   host_stats   host, 2 doubles: mean completion time, its standard error
  *   host_trials  host, [trials] completion times, or NULL
@@ -325,9 +328,9 @@ double nolo_expected_pair_exchange(double mu, double sigma);
  * NoLoCo a worker only waits for the n members of its random subgroup (the
  * same draw as nolo_outer_step, with step = outer iteration and boundary =
  * trial).  Reports the time for all workers to finish T outer iterations.
- *   seed    inner step k of worker w in outer iteration t of trial s uses
- *           philox4x64-10(counter = (k, w, t, 4), key = (seed, s)), transformed
- *           as in nolo_sim_tree_allreduce
+ *   seed    inner step k of worker w in outer iteration t of trial s is
+ *           position k % 4 of the block with counter (k / 4, w, t, 4) and key
+ *           (seed, s), transformed as in nolo_sim_tree_allreduce
  *   host_stats   host, 4 doubles: mean time with the global barrier, mean time
  *           with subgroup waits, then the standard errors of the two means
  *   host_trials  host, [trials][2] (barrier, subgroup) per trial, or NULL

@@ -7,8 +7,10 @@
 //  * straggler effect: inner-step times LogNormal(mu, sigma^2); DiLoCo waits at a global barrier
 //    after every H inner steps, NoLoCo only for the members of its random subgroup of n.
 //
-// Random numbers: Philox-4x64-10 words -> u = ((x >> 11) + 0.5) 2^-53 -> Box-Muller
-// z = sqrt(-2 ln u1) cos(2 pi u2) from words 0 and 1 -> t = exp(mu + sigma z).  float64 throughout.
+// Random numbers: every Philox-4x64-10 block yields four times.  Words -> u = ((x >> 11) + 0.5) 2^-53;
+// Box-Muller on the word pairs (0,1) and (2,3), r = sqrt(-2 ln u_a), gives the normals
+// [r01 cos, r01 sin, r23 cos, r23 sin] of the angle 2 pi u_b; t = exp(mu + sigma z).  Sample j of a
+// stream is position j % 4 of block j / 4.  float64 throughout.
 #include "nolo_internal.h"
 #include "nolo_philox.cuh"
 
@@ -24,9 +26,20 @@ __device__ __forceinline__ double uniform_open(uint64_t x) {
     return ((double)(x >> 11) + 0.5) * 0x1.0p-53;
 }
 
-__device__ __forceinline__ double lognormal(const Philox4& r, double mu, double sigma) {
-    const double z = sqrt(-2.0 * log(uniform_open(r.w0))) * cospi(2.0 * uniform_open(r.w1));
-    return exp(mu + sigma * z);
+// The two log-normal times of one word pair: cosine first, sine second.
+__device__ __forceinline__ void lognormal2(uint64_t wa, uint64_t wb, double mu, double sigma, double& t_cos,
+                                           double& t_sin) {
+    double s, c;
+    const double r = sqrt(-2.0 * log(uniform_open(wa)));
+    sincospi(2.0 * uniform_open(wb), &s, &c);
+    t_cos = exp(mu + sigma * (r * c));
+    t_sin = exp(mu + sigma * (r * s));
+}
+
+// The four log-normal times of one block.
+__device__ __forceinline__ void lognormal4(const Philox4& b, double mu, double sigma, double (&t)[4]) {
+    lognormal2(b.w0, b.w1, mu, sigma, t[0], t[1]);
+    lognormal2(b.w2, b.w3, mu, sigma, t[2], t[3]);
 }
 
 // Maximum over the CTA, returned to every thread.  Contains two barriers.
@@ -51,19 +64,30 @@ __global__ void tree_allreduce_kernel(int W, double mu, double sigma, uint64_t s
     const uint64_t trial = blockIdx.x;
     for (int i = threadIdx.x; i < 2 * W; i += blockDim.x) node[i] = 0.0;
     __syncthreads();
+    // A block serves the four nodes 4q .. 4q+3; two siblings 2p, 2p+1 share one of its word pairs.  One
+    // thread per sibling pair: the levels near the root have few nodes, so the work of a block is
+    // split over two threads (each recomputes the block's integer rounds) rather than halving the
+    // number of busy threads.
     for (int first = W >> 1; first >= 1; first >>= 1) {          // parents of one level: first .. 2*first-1
         for (int p = first + threadIdx.x; p < 2 * first; p += blockDim.x) {
-            const double a = node[2 * p] +
-                lognormal(philox4x64_10(2 * p, trial, 0, kDomainTree, seed, 0), mu, sigma);
-            const double b = node[2 * p + 1] +
-                lognormal(philox4x64_10(2 * p + 1, trial, 0, kDomainTree, seed, 0), mu, sigma);
-            node[p] = fmax(a, b);
+            const Philox4 b = philox4x64_10(p >> 1, trial, 0, kDomainTree, seed, 0);   // children 2p, 2p+1 are in block p/2
+            double ta, tb;
+            if (p & 1) lognormal2(b.w2, b.w3, mu, sigma, ta, tb);
+            else lognormal2(b.w0, b.w1, mu, sigma, ta, tb);
+            node[p] = fmax(node[2 * p] + ta, node[2 * p + 1] + tb);
         }
         __syncthreads();
     }
-    for (int first = 2; first < 2 * W; first <<= 1) {            // children of one level, top down
-        for (int c = first + threadIdx.x; c < 2 * first; c += blockDim.x)
-            node[c] = node[c >> 1] + lognormal(philox4x64_10(c, trial, 1, kDomainTree, seed, 0), mu, sigma);
+    for (int first = 2; first < 2 * W; first <<= 1) {            // children of one level, top down, in sibling pairs
+        for (int c = first + 2 * threadIdx.x; c < 2 * first; c += 2 * blockDim.x) {
+            const Philox4 b = philox4x64_10(c >> 2, trial, 1, kDomainTree, seed, 0);
+            double ta, tb;
+            if (c & 2) lognormal2(b.w2, b.w3, mu, sigma, ta, tb);
+            else lognormal2(b.w0, b.w1, mu, sigma, ta, tb);
+            const double parent = node[c >> 1];
+            node[c] = parent + ta;
+            node[c + 1] = parent + tb;
+        }
         __syncthreads();
     }
     double m = 0.0;
@@ -89,8 +113,13 @@ __global__ void straggler_kernel(int W, int n, int H, int T, double mu, double s
         double longest = 0.0;
         for (int w = threadIdx.x; w < W; w += blockDim.x) {
             double work = 0.0;
-            for (int k = 0; k < H; ++k)
-                work += lognormal(philox4x64_10(k, w, t, kDomainStraggler, seed, trial), mu, sigma);
+            for (int k0 = 0; k0 < H; k0 += 4) {                   // inner steps k0 .. k0+3 share a block
+                double step[4];
+                lognormal4(philox4x64_10(k0 >> 2, w, t, kDomainStraggler, seed, trial), mu, sigma, step);
+#pragma unroll
+                for (int l = 0; l < 4; ++l)
+                    if (k0 + l < H) work += step[l];
+            }
             longest = fmax(longest, work);
             done[w] = clock[w] + work;
             keys[w] = draw_key(w, trial, 0, kDomainGroups, seed, t);
