@@ -146,6 +146,30 @@ def test_nan_and_inf_propagate_within_their_subgroup_only(nolo, bf16):
     assert np.array_equal(got_phi[bad & ~np.isnan(want[0])], want[0][bad & ~np.isnan(want[0])])   # signed Inf
 
 
+@pytest.mark.parametrize("W,n", [(8, 2), (32, 16), (256, 128)])
+def test_infinite_slow_weight_stays_within_its_subgroup(nolo, W, n):
+    """An infinite phi (a replica that has already diverged) makes that parameter non-finite for
+    every member of its subgroup, as in the float64 definition, and touches nothing else.  Only
+    finiteness is compared there: Inf - Inf arises in both, in different places."""
+    P = 777
+    phi, theta, delta = synth.make_state(W, P, 31)
+    phi[1, 5] = float("inf")
+    phi[W - 1, 700] = float("-inf")
+    d = [x.cuda() for x in (phi, theta, delta)]
+    h = nolo.nolo_create(W, n, P, 1, *F)
+    nolo.nolo_bind_state(h, *d)
+    nolo.nolo_outer_step(h, 4, 4)
+    torch.cuda.synchronize()
+    perm = nolo.nolo_get_groups(h)
+    nolo.nolo_destroy(h)
+    want = O.outer_step(to_np(phi)[:, :P], to_np(theta)[:, :P], to_np(delta)[:, :P], perm, n, *F, O.THETA_F32)
+    for got, w in zip((to_np(d[0])[:, :P], to_np(d[2])[:, :P], to_np(d[1])[:, :P]), want):
+        assert np.array_equal(np.isfinite(got), np.isfinite(w))
+        bad = ~np.isfinite(w)
+        assert bad.sum() == 2 * n
+        assert_close_f32(np.where(bad, 0, got), np.where(bad, 0, w), "finite part")
+
+
 @pytest.mark.parametrize("W,n", [(4, 2), (8, 8), (24, 12), (72, 72), (130, 130), (200, 200), (600, 600)])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_guard_bands_around_every_buffer_stay_intact(nolo, W, n, bf16):
