@@ -643,6 +643,6 @@ const char* nolo_strerror(int status) {
 
 const char* nolo_last_error(nolo_handle* h) { return h ? h->err : ""; }
 
-int nolo_version(void) { return 100; }
+int nolo_version(void) { return 200; }
 
 }  // extern "C"

@@ -653,10 +653,9 @@ cudaError_t launch_group_mean(const float* phi, const int32_t* perm, int W, int 
     const double inv_n = 1.0 / (double)n;
     // rows of the means are 32-byte aligned when the base is (the stride is a multiple of 64 bytes)
     const bool wide = (reinterpret_cast<uintptr_t>(mean) & 31u) == 0;
-#define NOLO_MEAN_LAUNCH(I, WD) group_mean_kernel<I, WD><<<grid, kThreads, 0, stream>>>(phi, perm, n, stride, P, mean, mean_stride, inv_n)
-    if (items == 2) { if (wide) NOLO_MEAN_LAUNCH(2, true); else NOLO_MEAN_LAUNCH(2, false); }
-    else { if (wide) NOLO_MEAN_LAUNCH(1, true); else NOLO_MEAN_LAUNCH(1, false); }
-#undef NOLO_MEAN_LAUNCH
+    auto launch = [&](auto kernel) { kernel<<<grid, kThreads, 0, stream>>>(phi, perm, n, stride, P, mean, mean_stride, inv_n); };
+    if (items == 2) launch(wide ? group_mean_kernel<2, true> : group_mean_kernel<2, false>);
+    else launch(wide ? group_mean_kernel<1, true> : group_mean_kernel<1, false>);
     return cudaGetLastError();
 }
 
