@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import c_oracle as C
 from oracle import nolo_oracle as O
 from paper_2506_10911_b200 import synth
 from tests.helpers import assert_bf16_within_1ulp, assert_close_f32, to_np
@@ -68,11 +69,15 @@ def run_config(nolo, W, n, P, theta_dtype, hp, steps, drift="normal", seed0=0):
     h = nolo.nolo_create(W, n, P, 1, *hp)
     nolo.nolo_bind_state(h, phi, theta, delta)
     cols = sample_columns(P, W, seed0 + 17).to(dev)
+    # a sample sixteen times larger for the last step, judged by the C writing of the oracle
+    # (which has been cross-checked against the NumPy one and is fast enough for it)
+    wide = sample_columns(P, W, seed0 + 99, width=1 << 14, budget=1 << 25).to(dev)
     for k in range(steps):
         seed, step = seed0 + k, k
         if k:
             synth.apply_drift_(phi, theta, P, seed=1000 + seed, drift=drift)
         pre = [gather(x, cols) for x in (phi, theta, delta)]
+        pre_wide = [gather(x, wide) for x in (phi, theta, delta)] if k == steps - 1 else None
         probe = phi[:, P // 3: P // 3 + 4096].clone()          # a window the oracle does not look at
         nolo.nolo_outer_step(h, seed, step)
         torch.cuda.synchronize()
@@ -85,6 +90,14 @@ def run_config(nolo, W, n, P, theta_dtype, hp, steps, drift="normal", seed0=0):
             assert_bf16_within_1ulp(gather(theta, cols), want[2], f"theta step {k}")
         else:
             assert_close_f32(gather(theta, cols), want[2], f"theta step {k}")
+        if pre_wide is not None:
+            want = C.outer_step(pre_wide[0], pre_wide[1], pre_wide[2], perm, n, *hp, O.THETA_BF16 if bf16 else O.THETA_F32)
+            assert_close_f32(gather(phi, wide), want[0], f"phi step {k}, wide sample")
+            assert_close_f32(gather(delta, wide), want[1], f"delta step {k}, wide sample")
+            if bf16:
+                assert_bf16_within_1ulp(gather(theta, wide), want[2], f"theta step {k}, wide sample")
+            else:
+                assert_close_f32(gather(theta, wide), want[2], f"theta step {k}, wide sample")
         # whole-buffer properties
         assert not torch.equal(probe, phi[:, P // 3: P // 3 + 4096])
         for w in range(W):
