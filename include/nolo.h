@@ -168,6 +168,8 @@ int nolo_outer_step_prepared(nolo_handle* h, uint64_t seed, uint64_t step);
  *   err, err_len  optional host buffer that receives a message when the status is not NOLO_OK
  * The first call on each device looks up the array's device address (that device must be
  * current, as it must for every call); make that first call before any stream capture begins.
+ * At that first call the driver may also load the library's device code, as it does at any
+ * first launch, and take device memory for it once; no later call takes any.
  * All calls on a device share the one table and each call overwrites the entries it uses, so
  * nothing needs clearing between calls -- but two calls whose GPU work overlaps (different
  * streams, no ordering between them) race on the table and give undefined subgroups: order them.
