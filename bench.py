@@ -81,10 +81,10 @@ def kernel_name(n: int, theta: str) -> str:
     if n <= 8:
         items = 4 if n == 1 else (2 if (n == 2 and theta != "bf16") else 1)
         return f"outer_step_reg_kernel<{n},{t},{items}>"
-    if n <= 64:
-        return f"outer_step_split_kernel<{t}> (warps share the subgroup)"
-    shape = ("8 warps,32 quads,4 rows" if n <= 128 else "8 warps,32 quads,8 rows" if n <= 224 else
-             "8 warps,16 quads,8 rows" if n <= 640 else "16 warps,16 quads,8 rows")
+    shape = ("128 threads,128 quads,4 rows" if n <= 12 else "128 threads,64 quads,8 rows" if n <= 24 else
+             "256 threads,64 quads,4 rows" if n <= 64 else "256 threads,64 quads,8 rows" if n <= 96 else
+             "256 threads,32 quads,4 rows" if n <= 128 else "256 threads,32 quads,8 rows" if n <= 224 else
+             "256 threads,16 quads,8 rows" if n <= 640 else "512 threads,16 quads,8 rows")
     return f"outer_step_twopass_kernel<{t},{shape}> (second read of phi from L1/L2)"
 
 
@@ -416,7 +416,7 @@ def extra_configs(nolo, dev, peak, copy_gbs, args):
     for W in (8, 32, 128):
         run(W, 1 << 26, "f32", [(f"config 5: W={W} n={n} P=2^26 fp32, Student-t(3) drift", n, GAMMA, 3)
                                 for n in (2, 4, 8)], drift="student_t3")
-    for n in (16, 32, 64, 96, 128, 192, 256, 512, 1024):
+    for n in (9, 16, 32, 64, 96, 128, 192, 256, 512, 1024):
         for theta in ("f32", "bf16"):
             P = max(1 << 16, ((3 << 28) // n) & ~63)           # about 3.2e9 bytes of phi
             run(n, P, theta, [(f"large_n: one subgroup of n=W={n}, P={P}, {theta} theta (DiLoCo mode)", n, GAMMA, 5)])

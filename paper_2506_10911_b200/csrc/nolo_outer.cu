@@ -11,17 +11,16 @@
 //   phi_i'   = phi_i + delta_i'                                           (Eq. 3)
 //   theta_i' = phi_i'   (start of the next inner phase)
 //
-// Three kernels cover the subgroup sizes:
+// Two kernels cover the subgroup sizes:
 //   n <= 8        register-resident: one thread holds its quad of every member;
-//   8 < n <= 64   the members are shared out over the warps of one CTA, still in registers;
-//   n > 64        two passes over the members, the second read of phi served by L1/L2.
+//   n > 8         two passes over the members, the second read of phi served by L1/L2.
 //
 // Arithmetic.  Delta_j is formed per member and summed in float32 in short fixed-order partial
 // sums.  gamma * (phi_i - mean phi) is a small number formed from large ones: a mean rounded to
 // float32 would pass half an ulp of |phi| straight into delta', whose tolerance does not grow
 // with |phi|.  So the mean is carried as an unevaluated float32 pair hi + lo (about 46 bits):
 // the register kernel refines a float32 mean by the mean of the residuals phi_j - mean, the
-// other two sum phi with error-free additions (Knuth's two-sum: the rounding error of every
+// two-pass kernel sums phi with error-free additions (Knuth's two-sum: the rounding error of every
 // addition is recovered exactly and kept in lo).  Float64 accumulators would do the same, but
 // the float32 <-> float64 conversions they need run at 16 per clock per SM on B200 and cost
 // the wide-subgroup kernels 20-35 % of their bandwidth when measured.
@@ -268,130 +267,53 @@ outer_step_reg_kernel(const KArgs a) {
     if ((a.P & 3) && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) scalar_tail<ThetaT>(a, g);
 }
 
-// ---- 8 < n <= 64: the members shared out over the warps of one CTA ------------------------
+// ---- n > 8: two passes over the members, the second read of phi served by L1 / L2 ----------
 //
-// Holding phi of every member of a tile in registers costs n x 512 bytes per 32 quads, and the
-// kernel only streams at full bandwidth while more than one CTA fits on an SM (one CTA's loads
-// must overlap another's barrier and stores).  Warp w of the G <= 8 warps holds up to 8 members,
-// w*MPW .. w*MPW+MPW-1, for the same 32 quads (each member row is read in coalesced 512-byte
-// segments); the warps' partial sums meet in shared memory and are added in warp order, so the
-// result is deterministic and identical in every warp.  As in the small-n kernel every element
-// is read once and written once.  The shape (8 members per warp) measured best on B200 among
-// 4 and 8 per warp and CTAs of 32 / 64 / 128 members.
-constexpr int kSplitMaxMembers = 64;   // members one CTA holds
-constexpr int kSplitPref = 8;          // members per warp aimed at when the subgroup has more than 16 members
-constexpr int kSplitMaxWarps = kSplitMaxMembers / kSplitPref;
-
-// Registers per thread capped so that several CTAs fit an SM.
-template <int MPW>
-struct SplitShape {
-    static constexpr int kRegs = MPW <= 4 ? 80 : 128;
-    static constexpr int kMinBlocks = 65536 / (kSplitMaxWarps * 32 * kRegs);
-};
-
-template <int MPW, typename ThetaT>
-__global__ void __launch_bounds__(kSplitMaxWarps * 32, SplitShape<MPW>::kMinBlocks)
-outer_step_split_kernel(const KArgs a) {
-    __shared__ float4 part_D[kSplitMaxWarps][32];
-    __shared__ PairSum part_P[kSplitMaxWarps][32];
-    const int G = blockDim.x >> 5;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = blockIdx.y;
-    const int n = a.n;
-    const int64_t q = (int64_t)blockIdx.x * 32 + lane;
-    const bool ok = q < (a.P >> 2);
-    const int j0 = warp * MPW;
-
-    int row[MPW];
-#pragma unroll
-    for (int m = 0; m < MPW; ++m) row[m] = (j0 + m < n) ? __ldg(a.perm + g * n + j0 + m) : -1;
-
-    float4 phi[MPW], dlt[MPW];
-    float4 sD = f4_zero();
-    PairSum sP;
-    sP.clear();
-    if (ok) {
-        typename ThetaRaw<ThetaT>::type raw[MPW];
-#pragma unroll
-        for (int m = 0; m < MPW; ++m) {
-            if (row[m] >= 0) {
-                const int64_t off = (int64_t)row[m] * a.stride;
-                phi[m] = __ldcs(reinterpret_cast<const float4*>(a.phi + off) + q);
-                raw[m] = load_theta_raw(static_cast<const ThetaT*>(a.theta) + off, q);
-            }
-        }
-#pragma unroll
-        for (int m = 0; m < MPW; ++m) {
-            if (row[m] >= 0)
-                dlt[m] = __ldcs(reinterpret_cast<const float4*>(a.delta + (int64_t)row[m] * a.stride) + q);
-        }
-#pragma unroll
-        for (int m = 0; m < MPW; ++m) {
-            if (row[m] >= 0) {
-                f4_add(sD, f4_sub(phi[m], widen(raw[m])));          // Eq. 1
-                sP.add(phi[m]);
-            }
-        }
-    }
-    part_D[warp][lane] = sD;
-    part_P[warp][lane] = sP;
-    __syncthreads();
-    if (ok) {
-        // sum over the warps of this CTA, in warp order
-        sD = part_D[0][lane];
-        sP = part_P[0][lane];
-        for (int w = 1; w < G; ++w) {
-            f4_add(sD, part_D[w][lane]);
-            sP.add(part_P[w][lane]);
-        }
-        if (a.mean_phi) sP = load_prepared_mean(a, g, q);
-        else sP.divide(a);
-#pragma unroll
-        for (int m = 0; m < MPW; ++m) {
-            if (row[m] >= 0)
-                update_store<ThetaT>(a, (int64_t)row[m] * a.stride, q, phi[m], sP.deviation(phi[m]), dlt[m], sD);
-        }
-    }
-    if ((a.P & 3) && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) scalar_tail<ThetaT>(a, g);
-}
-
-// ---- n > 64: two passes over the members, the second read of phi served by L1 / L2 ---------
-//
-// One CTA owns one subgroup x ROWQ quads.  Its threads form WARPS*32/ROWQ slots of ROWQ lanes;
-// slot s walks members s, s + SLOTS, ... in chunks of U rows in flight.  Pass 1 reads phi and
-// theta and accumulates the two sums; the slots' partial sums meet in shared memory; pass 2
-// reads phi again together with delta and writes the update.  Between the two reads of a phi
-// element lie only the other rows of the same CTA's tile (n x ROWQ x 16 bytes), so the second
+// One CTA owns one subgroup x ROWQ quads.  Its THREADS threads form THREADS/ROWQ slots of ROWQ
+// consecutive quads; slot s walks members s, s + SLOTS, ... in chunks of U rows in flight.  Pass 1
+// reads phi and theta and accumulates the two sums; the slots' partial sums meet in shared memory;
+// pass 2 reads phi again together with delta and writes the update.  Between the two reads of a
+// phi element lie only the other rows of the same CTA's tile (n x ROWQ x 16 bytes), so the second
 // read is served by L1 or L2 as long as the tiles of all resident CTAs fit there: profiled DRAM
 // traffic equals the algorithmic 24 / 20 bytes per worker-parameter, and nothing has to be parked
 // in registers or shared memory, whatever n is.  The first chunk of pass 2 depends on no sum, so
 // its loads are issued before the partial sums meet and are in flight across the CTA barrier.
-// No bulk copies, no clusters and no waits other than that one barrier.
+// No bulk copies, no clusters and no waits other than that one barrier (none at all with one slot).
 //
-// The shape trades three things: bytes in flight (warps x U), the width of a row segment (DRAM
-// likes 512 bytes better than 256) and the L2 footprint of the resident tiles
+// The shape trades three things: bytes in flight (threads x U), the width of the piece of a row
+// that one CTA streams (ROWQ x 16 bytes: DRAM likes 1-2 KB pieces better than 512-byte ones, and
+// 256-byte ones least) and the L2 footprint of the resident tiles
 // (CTAs per SM x n x ROWQ x 16 bytes x 148 SMs), which must stay well below the 126 MB of L2 or
-// the re-read goes to DRAM.  Measured best on B200 (fraction of a plain copy, float32 / bfloat16
-// theta): 8 warps x 32 quads x 4 rows, 3 CTAs per SM up to 128 members (0.94); 8 rows in flight
-// and 2 CTAs per SM up to 224 (0.92 - 0.90); 16-quad segments up to 640 (0.93 - 0.88); above that
-// 16 warps x 16 quads x 8 rows, one CTA per SM (0.92 - 0.84 at 1024).  Tried and measured slower on
-// this access pattern: rings of asynchronous copies (cp.async) that keep several chunks in
-// flight per thread (same rate: the kernel is not short of loads in flight), phi parked in shared
-// memory, and phi parked in tensor memory (tcgen05.st / tcgen05.ld; exact, but two CTAs of eight
-// warps per SM are too few warps: 0.78 - 0.85).  Even with the re-read of phi left out altogether
-// the same loops reach only 0.92 / 0.91 / 0.89 of a plain copy at n = 128 / 256 / 1024: what is lost is
-// lost to streaming n x 3 rows in 512-byte pieces, not to the second read.
-template <typename ThetaT, int WARPS, int ROWQ, int U, int MINB>
-__global__ void __launch_bounds__(WARPS * 32, MINB)
+// the re-read goes to DRAM.  Small subgroups therefore take wide pieces and few slots, large
+// ones narrow pieces; the best shapes have SLOTS x U close to n, so that a slot walks its rows
+// in one to four chunks.  Measured on B200 as a fraction of a plain copy (float32 / bfloat16
+// theta): 0.96-0.97 / 0.95-0.96 up to 48 members, 0.95 / 0.94 at 64 and at 96, 0.93 at 128,
+// 0.92-0.91 up to 224, 0.93-0.86 up to 640, 0.87 / 0.79 at 1024.
+//
+// Tried and measured slower on this access pattern: members held in registers by the warps of a
+// CTA, one pass (0.94 for 9-64 members: 512-byte pieces); rings of asynchronous copies (cp.async)
+// that keep several chunks in flight per thread (same rate: the kernel is not short of loads in
+// flight); phi parked in shared memory; phi parked in tensor memory (tcgen05.st / tcgen05.ld;
+// exact, but two CTAs of eight warps per SM are too few warps: 0.78-0.85); a persistent grid
+// (0.5-0.7: all CTAs in the same phase at once).  With the re-read of phi left out altogether
+// the 512-byte-piece loops reach only 0.92 / 0.91 / 0.89 of a plain copy at n = 128 / 256 / 1024:
+// what is lost is lost to streaming n x 3 rows in narrow pieces, not to the second read.
+template <typename ThetaT, int THREADS, int ROWQ, int U, int MINB>
+__global__ void __launch_bounds__(THREADS, MINB)
 outer_step_twopass_kernel(const KArgs a) {
-    constexpr int SLOTS = WARPS * 32 / ROWQ;
-    constexpr int SPW = 32 / ROWQ;            // slots per warp
-    static_assert(ROWQ == 32 || ROWQ == 16 || ROWQ == 8, "a slot is a whole fraction of a warp");
-    __shared__ float4 part_D[WARPS][ROWQ];
-    __shared__ PairSum part_P[WARPS][ROWQ];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ql = lane % ROWQ;
-    const int slot = warp * SPW + lane / ROWQ;
+    static_assert(THREADS % 32 == 0 && THREADS % ROWQ == 0, "slots tile the CTA");
+    static_assert(ROWQ >= 32 ? ROWQ % 32 == 0 : 32 % ROWQ == 0, "a slot is whole warps or a whole fraction of one");
+    constexpr int SLOTS = THREADS / ROWQ;
+    constexpr int WARPS = THREADS / 32;
+    // Partial sums that meet in shared memory: one per slot when slots are whole warps, one per warp
+    // when a warp holds several slots (those are first added by shuffles).
+    constexpr int PARTS = ROWQ >= 32 ? SLOTS : WARPS;
+    __shared__ float4 part_D[PARTS][ROWQ];
+    __shared__ PairSum part_P[PARTS][ROWQ];
+    const int lane = threadIdx.x & 31;
+    const int ql = threadIdx.x % ROWQ;
+    const int slot = threadIdx.x / ROWQ;
+    const int part = ROWQ >= 32 ? slot : (threadIdx.x >> 5);
     const int g = blockIdx.y;
     const int n = a.n;
     const int32_t* members = a.perm + (int64_t)g * n;
@@ -438,41 +360,48 @@ outer_step_twopass_kernel(const KArgs a) {
         }
     };
     if (ok) load_chunk(slot);      // in flight while the partial sums meet
-    // the slots of one warp that share a quad (fixed order), then the warps through shared memory
+    if constexpr (ROWQ < 32) {
+        // the slots of one warp that share a quad, in a fixed order
 #pragma unroll
-    for (int o = ROWQ; o < 32; o <<= 1) {
-        PairSum t;
-        float4 d;
-        d.x = __shfl_xor_sync(0xffffffffu, sD.x, o); d.y = __shfl_xor_sync(0xffffffffu, sD.y, o);
-        d.z = __shfl_xor_sync(0xffffffffu, sD.z, o); d.w = __shfl_xor_sync(0xffffffffu, sD.w, o);
-        t.hi.x = __shfl_xor_sync(0xffffffffu, sP.hi.x, o); t.hi.y = __shfl_xor_sync(0xffffffffu, sP.hi.y, o);
-        t.hi.z = __shfl_xor_sync(0xffffffffu, sP.hi.z, o); t.hi.w = __shfl_xor_sync(0xffffffffu, sP.hi.w, o);
-        t.lo.x = __shfl_xor_sync(0xffffffffu, sP.lo.x, o); t.lo.y = __shfl_xor_sync(0xffffffffu, sP.lo.y, o);
-        t.lo.z = __shfl_xor_sync(0xffffffffu, sP.lo.z, o); t.lo.w = __shfl_xor_sync(0xffffffffu, sP.lo.w, o);
-        // both partners add (lower slot) + (higher slot) in that order, so they agree bit for bit
-        if (lane & o) {
-            PairSum mine = sP;
-            sP = t;
-            sP.add(mine);
-            d.x += sD.x; d.y += sD.y; d.z += sD.z; d.w += sD.w;
-            sD = d;
-        } else {
-            sP.add(t);
-            f4_add(sD, d);
+        for (int o = ROWQ; o < 32; o <<= 1) {
+            PairSum t;
+            float4 d;
+            d.x = __shfl_xor_sync(0xffffffffu, sD.x, o); d.y = __shfl_xor_sync(0xffffffffu, sD.y, o);
+            d.z = __shfl_xor_sync(0xffffffffu, sD.z, o); d.w = __shfl_xor_sync(0xffffffffu, sD.w, o);
+            t.hi.x = __shfl_xor_sync(0xffffffffu, sP.hi.x, o); t.hi.y = __shfl_xor_sync(0xffffffffu, sP.hi.y, o);
+            t.hi.z = __shfl_xor_sync(0xffffffffu, sP.hi.z, o); t.hi.w = __shfl_xor_sync(0xffffffffu, sP.hi.w, o);
+            t.lo.x = __shfl_xor_sync(0xffffffffu, sP.lo.x, o); t.lo.y = __shfl_xor_sync(0xffffffffu, sP.lo.y, o);
+            t.lo.z = __shfl_xor_sync(0xffffffffu, sP.lo.z, o); t.lo.w = __shfl_xor_sync(0xffffffffu, sP.lo.w, o);
+            // both partners add (lower slot) + (higher slot) in that order, so they agree bit for bit
+            if (lane & o) {
+                PairSum mine = sP;
+                sP = t;
+                sP.add(mine);
+                d.x += sD.x; d.y += sD.y; d.z += sD.z; d.w += sD.w;
+                sD = d;
+            } else {
+                sP.add(t);
+                f4_add(sD, d);
+            }
         }
     }
-    if (lane < ROWQ) {
-        part_D[warp][ql] = sD;
-        part_P[warp][ql] = sP;
+    if constexpr (PARTS > 1) {
+        // the partial sums of the slots (or warps) meet in shared memory
+        if (ROWQ >= 32 || lane < ROWQ) {
+            part_D[part][ql] = sD;
+            part_P[part][ql] = sP;
+        }
+        __syncthreads();
     }
-    __syncthreads();
     if (ok) {
-        sD = part_D[0][ql];
-        sP = part_P[0][ql];
+        if constexpr (PARTS > 1) {          // added in index order: the same result in every slot
+            sD = part_D[0][ql];
+            sP = part_P[0][ql];
 #pragma unroll
-        for (int w = 1; w < WARPS; ++w) {
-            f4_add(sD, part_D[w][ql]);
-            sP.add(part_P[w][ql]);
+            for (int w = 1; w < PARTS; ++w) {
+                f4_add(sD, part_D[w][ql]);
+                sP.add(part_P[w][ql]);
+            }
         }
         if (a.mean_phi) sP = load_prepared_mean(a, g, q);
         else sP.divide(a);
@@ -582,26 +511,23 @@ cudaError_t launch_reg(const KArgs& k, int groups, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
-template <int MPW, typename ThetaT>
-cudaError_t launch_split(const KArgs& k, int groups, int warps, cudaStream_t stream) {
-    dim3 grid;
-    if (!tile_grid(k, 32, groups, &grid)) return cudaErrorInvalidConfiguration;
-    outer_step_split_kernel<MPW, ThetaT><<<grid, warps * 32, 0, stream>>>(k);
-    return cudaGetLastError();
-}
-
-template <typename ThetaT, int WARPS, int ROWQ, int U, int MINB>
+template <typename ThetaT, int THREADS, int ROWQ, int U, int MINB>
 cudaError_t launch_twopass(const KArgs& k, int groups, cudaStream_t stream) {
     dim3 grid;
     if (!tile_grid(k, ROWQ, groups, &grid)) return cudaErrorInvalidConfiguration;
-    outer_step_twopass_kernel<ThetaT, WARPS, ROWQ, U, MINB><<<grid, WARPS * 32, 0, stream>>>(k);
+    outer_step_twopass_kernel<ThetaT, THREADS, ROWQ, U, MINB><<<grid, THREADS, 0, stream>>>(k);
     return cudaGetLastError();
 }
 
-// Subgroup sizes up to which each two-pass shape is used (by measurement, see the kernel's comment).
-constexpr int kTwoPassMaxN4Rows = 128;   // 8 warps x 32 quads x 4 rows in flight, 3 CTAs per SM
-constexpr int kTwoPassMaxN32Quads = 224; // 8 warps x 32 quads x 8 rows, 2 CTAs per SM
-constexpr int kTwoPassMaxN8Warps = 640;  // 8 warps x 16 quads x 8 rows, 2 CTAs per SM; above: 16 warps, 1 CTA per SM
+// Subgroup sizes up to which each two-pass shape is used (by measurement, see the kernel's comment):
+// threads x quads per row piece x rows in flight per slot, CTAs per SM.
+constexpr int kTwoPassMaxN1Slot = 12;     // 128 x 128 x 4, 6 CTAs: one slot, no barrier
+constexpr int kTwoPassMaxN2Slots = 24;    // 128 x 64 x 8, 4 CTAs
+constexpr int kTwoPassMaxN64Quads4 = 64;  // 256 x 64 x 4, 3 CTAs
+constexpr int kTwoPassMaxN64Quads8 = 96;  // 256 x 64 x 8, 2 CTAs
+constexpr int kTwoPassMaxN4Rows = 128;    // 256 x 32 x 4, 3 CTAs
+constexpr int kTwoPassMaxN32Quads = 224;  // 256 x 32 x 8, 2 CTAs
+constexpr int kTwoPassMaxN8Warps = 640;   // 256 x 16 x 8, 2 CTAs; above: 512 x 16 x 8, 1 CTA
 
 template <typename ThetaT>
 cudaError_t dispatch(const KArgs& k, int groups, cudaStream_t stream) {
@@ -617,25 +543,14 @@ cudaError_t dispatch(const KArgs& k, int groups, cudaStream_t stream) {
         case 8:  return launch_reg<8, ThetaT, 1>(k, groups, stream);
         default: break;
     }
-    if (k.n <= kSplitMaxMembers) {
-        const int pref = k.n > 16 ? kSplitPref : 4;                        // members per warp aimed at
-        const int G = (k.n + pref - 1) / pref;                             // warps
-        const int mpw = (k.n + G - 1) / G;                                 // members per warp
-        switch (mpw) {
-            case 1: return launch_split<1, ThetaT>(k, groups, G, stream);
-            case 2: return launch_split<2, ThetaT>(k, groups, G, stream);
-            case 3: return launch_split<3, ThetaT>(k, groups, G, stream);
-            case 4: return launch_split<4, ThetaT>(k, groups, G, stream);
-            case 5: return launch_split<5, ThetaT>(k, groups, G, stream);
-            case 6: return launch_split<6, ThetaT>(k, groups, G, stream);
-            case 7: return launch_split<7, ThetaT>(k, groups, G, stream);
-            default: return launch_split<8, ThetaT>(k, groups, G, stream);
-        }
-    }
-    if (k.n <= kTwoPassMaxN4Rows) return launch_twopass<ThetaT, 8, 32, 4, 3>(k, groups, stream);
-    if (k.n <= kTwoPassMaxN32Quads) return launch_twopass<ThetaT, 8, 32, 8, 2>(k, groups, stream);
-    if (k.n <= kTwoPassMaxN8Warps) return launch_twopass<ThetaT, 8, 16, 8, 2>(k, groups, stream);
-    return launch_twopass<ThetaT, 16, 16, 8, 1>(k, groups, stream);
+    if (k.n <= kTwoPassMaxN1Slot) return launch_twopass<ThetaT, 128, 128, 4, 6>(k, groups, stream);
+    if (k.n <= kTwoPassMaxN2Slots) return launch_twopass<ThetaT, 128, 64, 8, 4>(k, groups, stream);
+    if (k.n <= kTwoPassMaxN64Quads4) return launch_twopass<ThetaT, 256, 64, 4, 3>(k, groups, stream);
+    if (k.n <= kTwoPassMaxN64Quads8) return launch_twopass<ThetaT, 256, 64, 8, 2>(k, groups, stream);
+    if (k.n <= kTwoPassMaxN4Rows) return launch_twopass<ThetaT, 256, 32, 4, 3>(k, groups, stream);
+    if (k.n <= kTwoPassMaxN32Quads) return launch_twopass<ThetaT, 256, 32, 8, 2>(k, groups, stream);
+    if (k.n <= kTwoPassMaxN8Warps) return launch_twopass<ThetaT, 256, 16, 8, 2>(k, groups, stream);
+    return launch_twopass<ThetaT, 512, 16, 8, 1>(k, groups, stream);
 }
 
 }  // namespace

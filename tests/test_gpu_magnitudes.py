@@ -57,7 +57,7 @@ def step_and_compare(nolo, W, n, P, theta_dtype, hp, seed, prepared=False):
 
 
 # one subgroup size per dispatch path and per boundary between paths
-SIZES = [1, 2, 3, 4, 8, 9, 24, 48, 64, 65, 96, 112, 113, 128, 129, 192, 224, 225, 256, 257, 300, 512, 640, 641, 1024]
+SIZES = [1, 2, 3, 4, 8, 9, 12, 13, 24, 25, 48, 64, 65, 96, 97, 112, 128, 129, 192, 224, 225, 256, 257, 300, 512, 640, 641, 1024]
 
 
 @pytest.mark.parametrize("n", SIZES)

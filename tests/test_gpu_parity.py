@@ -85,13 +85,13 @@ def test_group_sizes_and_ragged_tiles(nolo, n, bf16):
     run_both(nolo, W, n, 5 * 1024 + 3, 7, 3, dt, stride=5 * 1024 + 16)
 
 
-@pytest.mark.parametrize("n", [5, 6, 7, 9, 16, 17, 24, 32, 33, 48, 49, 64, 65, 96, 97, 100, 112, 113, 128, 129, 160, 192, 193, 224, 225, 256, 300,
-                               512, 520, 640, 641])
+@pytest.mark.parametrize("n", [5, 6, 7, 9, 10, 12, 13, 16, 17, 24, 25, 32, 33, 48, 49, 64, 65, 96, 97, 100, 112, 113, 128, 129, 160, 192, 193, 224,
+                               225, 256, 300, 512, 520, 640, 641])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_large_subgroups(nolo, n, bf16):
-    """8 < n <= 64 runs the kernel that shares the members out over the warps of a CTA (with
-    masked member slots when n does not fill them); above that the two-pass kernel in its four
-    shapes (up to 128, 224 and 640 members, and beyond).  Two subgroups, ragged P."""
+    """n > 8 runs the two-pass kernel in its eight shapes (up to 12, 24, 64, 96, 128, 224 and 640
+    members, and beyond; slots of one to four warps or of half a warp, with member slots masked
+    when n does not fill them).  Two subgroups, ragged P."""
     dt = torch.bfloat16 if bf16 else torch.float32
     run_both(nolo, 2 * n, n, 1000 + 3, 11, 4, dt)
     if n in (16, 100, 128):
@@ -171,11 +171,11 @@ def test_infinite_slow_weight_stays_within_its_subgroup(nolo, W, n):
         assert_close_f32(np.where(bad, 0, got), np.where(bad, 0, w), "finite part")
 
 
-@pytest.mark.parametrize("W,n", [(4, 2), (8, 8), (24, 12), (72, 72), (130, 130), (200, 200), (600, 600)])
+@pytest.mark.parametrize("W,n", [(4, 2), (8, 8), (24, 12), (40, 20), (64, 32), (72, 72), (130, 130), (200, 200), (600, 600), (700, 700)])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_guard_bands_around_every_buffer_stay_intact(nolo, W, n, bf16):
     """Each state tensor sits between two 4 KiB bands of a known pattern inside a larger
-    allocation; no kernel path (register-resident, warp-split, two-pass, ragged tail)
+    allocation; no kernel path (register-resident, two-pass in its shapes, ragged tail)
     may write outside its rows."""
     P, stride, band = 1000 + 3, 1008, 1024            # band in elements
     dt = torch.bfloat16 if bf16 else torch.float32

@@ -24,7 +24,7 @@ def nolo():
     return binding
 
 
-@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 8, 12, 64, 96, 160, 256, 384])
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 8, 12, 20, 40, 64, 96, 128, 160, 256, 384, 700])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_prepared_step_matches_oracle(nolo, n, bf16):
     W = 2 * n if n <= 256 else n
