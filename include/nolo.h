@@ -108,7 +108,7 @@ int nolo_bind_state(nolo_handle* h, void* phi, void* theta, void* delta,
  * that gamma (phi_i - mean) is accurate for weights of any magnitude; sums in a
  * fixed order (results are reproducible bit for bit); every element of every
  * worker is fetched from device memory once and written once (subgroups of
- * more than 64 members request phi a second time, which the caches serve).
+ * more than 8 members request phi a second time, which the caches serve).
  * NaN and Inf are not special-cased: they make the same parameter of every
  * member of the subgroup non-finite and touch nothing else.
  * Asynchronous.  Errors: NOLO_EINVAL (NULL handle), NOLO_ESTATE (no state
