@@ -287,8 +287,8 @@ outer_step_reg_kernel(const KArgs a) {
 // the re-read goes to DRAM.  Small subgroups therefore take wide pieces and few slots, large
 // ones narrow pieces; the best shapes have SLOTS x U close to n, so that a slot walks its rows
 // in one to four chunks.  Measured on B200 as a fraction of a plain copy (float32 / bfloat16
-// theta): 0.96-0.97 / 0.95-0.96 up to 48 members, 0.95 / 0.94 at 64 and at 96, 0.93 at 128,
-// 0.92-0.91 up to 224, 0.93-0.86 up to 640, 0.87 / 0.79 at 1024.
+// theta): 0.96-0.97 / 0.94-0.96 up to 48 members, 0.95 / 0.94 at 64 and at 96, 0.93 at 128,
+// 0.92 up to 224, 0.93-0.88 up to 640, 0.89 / 0.84 at 1024.
 //
 // Tried and measured slower on this access pattern: members held in registers by the warps of a
 // CTA, one pass (0.94 for 9-64 members: 512-byte pieces); rings of asynchronous copies (cp.async)
