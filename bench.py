@@ -297,7 +297,7 @@ def run_reference(args):
     cores = host_cores()
     probe = oracle_sample_state(wl, sh, 1 << 16)
     t_probe = min(oracle_step(wl, probe, 0, cores) for _ in range(2)) / (1 << 16)   # seconds per column
-    budget = 120.0 / max(1, args.steps + args.warmup)
+    budget = args.ref_seconds / max(1, args.steps + args.warmup)
     cols = int(min(1 << 24, max(1 << 12, budget / t_probe)))
     state = oracle_sample_state(wl, sh, cols)
     for k in range(args.warmup):
@@ -688,6 +688,8 @@ def main():
     ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration records")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-cols", type=int, default=1 << 25)
+    ap.add_argument("--ref-seconds", type=float, default=120.0,
+                    help="--impl reference: CPU time the whole run (warm-up + steps) is sized for")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup)
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
